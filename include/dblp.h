@@ -1,0 +1,219 @@
+/*
+ * dblp.h -- C ABI of libdblp: the receive-side data path of the Dynamic Bounded-Loss Protocol (DBLP)
+ * for W simulated workers whose gradients are resident on one CUDA device (sm_100a).
+ *
+ * One communication round is four calls on one stream:
+ *
+ *   dblp_packetize   gradients            -> header ring + payload ring      (Algorithm 1, first step)
+ *   dblp_apply_loss  seeded loss process  -> delivered bitmap + arrival list (Sections II-C, V-B; property 1)
+ *   dblp_aggregate   arrival list + rings -> received bitmap + aggregate     (Algorithm 2; Algorithm 3 "mean")
+ *   dblp_check_bound received bitmap      -> per-worker loss counts, stop / continue decision (Section III-B)
+ *
+ * Conventions
+ *   - Every function returns DBLP_OK (0) or a negative dblp_status_t; nothing throws, aborts or traps.
+ *     dblp_last_error() gives the text of the calling thread's most recent failure.
+ *   - Unless an argument is marked HOST it is a DEVICE pointer owned by the caller, on the device that was
+ *     current when the plan was created.  The library allocates device memory only in dblp_plan_create.
+ *   - Per-round calls only enqueue work on the given stream (a cudaStream_t passed as void*; NULL = the
+ *     legacy default stream) and do not synchronise.  Counts that a later step needs stay on the device.
+ *   - Anomalies found on the device (bad slot index, header that contradicts the plan, wrong round, repeated
+ *     packet) are counted in dblp_counters_t and skipped; they never fault.
+ *   - Alignment: ring and aggregate base pointers 16-byte aligned; payload_bytes a multiple of 16.
+ *     Tensor sizes need no alignment (ragged edges take a scalar path).
+ *   - Limits: W * C < 2^31 packets per round, ring slots < 2^32 - 1, payload_bytes <= 65536.
+ */
+#ifndef DBLP_H
+#define DBLP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DBLP_OK = 0,
+    DBLP_EINVAL = -1,    /* null pointer, zero size, value out of range */
+    DBLP_EALIGN = -2,    /* pointer or payload size not 16-byte aligned */
+    DBLP_ECAPACITY = -3, /* a limit above is exceeded, or the workspace is too small */
+    DBLP_ECUDA = -4,     /* a CUDA runtime call failed; text in dblp_last_error() */
+    DBLP_ETIMEOUT = -5   /* reserved: no call in this library waits on the device */
+} dblp_status_t;
+
+typedef enum { DBLP_F32 = 0, DBLP_BF16 = 1 } dblp_dtype_t;
+typedef enum { DBLP_LOSS_NONE = 0, DBLP_LOSS_IID = 1, DBLP_LOSS_GE = 2, DBLP_LOSS_MICROBURST = 3 } dblp_loss_kind_t;
+enum { DBLP_SUM = 0, DBLP_MEAN = 1 }; /* flags of dblp_aggregate */
+
+/* Packet header, 32 bytes, stored beside (not inside) the payload.  seq, round and len_bytes are the paper's
+ * three fields (Section IV-A); tensor_id and offset_elems are the id/offset tags of the prior work the paper
+ * builds on (Section III-A), redundant with seq given the plan and verified against it on receipt; worker stands
+ * for the per-worker UDP port (Section IV-D). */
+typedef struct {
+    uint32_t seq;          /* unique per (worker, round), 0 .. C-1 */
+    uint32_t round;        /* communication round the packet was sent in */
+    uint32_t len_bytes;    /* valid payload bytes (the last chunk of a tensor is short) */
+    uint32_t tensor_id;    /* index into the plan's tensor list */
+    uint64_t offset_elems; /* first element of the chunk inside its tensor */
+    uint32_t worker;       /* 0 .. W-1 */
+    uint32_t reserved;     /* written as 0 */
+} dblp_hdr_t;
+
+/* Loss process in integers: a packet's 32-bit draw u drops it iff u < threshold, thresholds in [0, 2^32].
+ * The paper injects loss without naming a generator (Sections II-C, V-B); the processes are:
+ *   IID         drop iff u0 < t_drop.
+ *   MICROBURST  one window of window_len consecutive sequence numbers, the same for every worker;
+ *               drop iff u0 < (inside ? t_drop_in : t_drop_out).
+ *   GE          two-state chain per worker in seq order: starts Bad iff u_init < t_init_bad; drop iff
+ *               u0 < (Bad ? t_drop_bad : t_drop_good); then Bad -> Good iff u1 < t_bg, Good -> Bad iff u1 < t_gb.
+ * Draws are Philox4x32-10 with key = seed and counter = (id low, id high, stream | attempt << 8, round),
+ * id = worker * C + seq. */
+typedef struct {
+    uint32_t kind; /* dblp_loss_kind_t */
+    uint32_t pad;
+    uint64_t t_drop;
+    uint64_t t_gb, t_bg, t_init_bad;
+    uint64_t t_drop_good, t_drop_bad;
+    uint64_t window_len;
+    uint64_t t_drop_in, t_drop_out;
+} dblp_loss_model_t;
+
+/* Receiver statistics of a round (device memory; all fields accumulate until dblp_round_reset). */
+typedef struct {
+    uint64_t n_arrived;  /* arrival-list entries examined */
+    uint64_t n_accepted; /* packets whose bit was newly set */
+    uint64_t n_dup;      /* valid packets of this round whose chunk had already arrived */
+    uint64_t n_stale;    /* valid packets of another round (Section III-A: dropped) */
+    uint64_t n_invalid;  /* slot outside the ring, or header contradicting the plan (Algorithm 2 integrity check) */
+    uint32_t status;     /* bit 0: arrival numbers exceeded 32 bits */
+    uint32_t pad;
+} dblp_counters_t;
+
+typedef struct dblp_plan dblp_plan_t;
+
+/* ---- plan: the constants exchanged once before training (Section IV-A) -------------------------------------
+ * tensor_numel (HOST, T values > 0): elements of each gradient tensor in flat order.  Chunking is per tensor:
+ * tensor t yields ceil(n_t / E) chunks, E = payload_bytes / element size; C is their total.
+ * bucket_seq_bounds (HOST, B+1 ascending sequence numbers from 0 to C, or NULL with B = 1): the ranges over
+ * which dblp_check_bound counts; one bucket is the paper's single bitmap per worker stream.
+ * Allocates the plan's device tables on the current device; *out is owned by the caller until dblp_plan_destroy. */
+int dblp_plan_create(const uint64_t* tensor_numel, uint32_t T, int dtype, uint32_t payload_bytes, uint32_t W,
+                     const uint64_t* bucket_seq_bounds, uint32_t B, dblp_plan_t** out);
+int dblp_plan_destroy(dblp_plan_t* plan);
+/* C = chunks per worker, N = elements per worker, M = W * C, row_words = ceil(C / 32) words per bitmap row.
+ * Any out pointer may be NULL. */
+int dblp_plan_query(const dblp_plan_t* plan, uint64_t* C, uint64_t* N, uint64_t* M, uint64_t* row_words);
+/* Bytes of scratch that dblp_apply_loss needs (the other calls need none). */
+int dblp_workspace_bytes(const dblp_plan_t* plan, size_t* bytes);
+
+/* HOST helper: rates -> thresholds floor(prob * 2^32).  IID uses mean_loss.  GE is the simple Gilbert chain
+ * (every packet sent in Bad is lost): P(Bad->Good) = 1 / mean_burst_len, P(Good->Bad) chosen so the stationary loss
+ * is mean_loss, start state drawn from the stationary law.  MICROBURST: window_len = ceil(window_frac * C). */
+int dblp_loss_model_from_rates(int kind, double mean_loss, double mean_burst_len, double window_frac, double p_in,
+                               double p_out, uint64_t C, dblp_loss_model_t* out);
+
+/* ---- packetize (Algorithm 1 "split data into chunks"; Sections IV-A, IV-B) ----------------------------------
+ * grads: HOST array of W device pointers, each a flat gradient of N elements of the plan's dtype (element-aligned).
+ * Writes M headers to hdr_ring and M payload slots of payload_bytes each to payload_ring; packet (w, seq) goes to
+ * slot w * C + seq; bytes of a slot past len_bytes are written as zero.  Rings may hold more than M slots (the
+ * rest is untouched). */
+int dblp_packetize(const dblp_plan_t* plan, const void* const* grads, uint32_t round, dblp_hdr_t* hdr_ring,
+                   void* payload_ring, void* stream);
+
+/* ---- apply_loss: which packets survive, and in which order they arrive ---------------------------------------
+ * model: HOST.  delivered_bits: W rows of row_words u32, bit (seq % 32) of word (seq / 32) set iff packet
+ * (w, seq) survives; padding bits zero.  arrival: capacity M u32; receives the surviving slot numbers in the order
+ * pi(0), pi(1), ... where pi is a seeded permutation of [0, M) (4-round Feistel network on the smallest even
+ * number of bits covering M, cycle-walked; round function = one Philox draw).  *n_arrived_dev (u64) = their count.
+ * ws: scratch of at least dblp_workspace_bytes(); contents need not be preserved between calls. */
+int dblp_apply_loss(const dblp_plan_t* plan, const dblp_loss_model_t* model, uint64_t seed, uint32_t round,
+                    uint32_t attempt, uint32_t* delivered_bits, uint32_t* arrival, uint64_t* n_arrived_dev, void* ws,
+                    size_t ws_bytes, void* stream);
+
+/* ---- aggregate = bookkeeping + masked reduce ------------------------------------------------------------------
+ * dblp_aggregate_book (Algorithm 2, chunk branch; Section III-A round filter): examines arrival[0 .. *n_arrived_dev)
+ * (at most arrival_cap entries).  An entry is invalid if its slot >= n_slots or its header contradicts the plan
+ * (worker < W, tensor_id < T, offset on a chunk boundary inside the tensor, len_bytes = that chunk's length,
+ * seq = that chunk's number); stale if header.round != round; otherwise it claims cell (worker, seq) of slot_key.
+ * slot_key: W * C u64, all-ones = nothing arrived yet, else (arrival number << 32) | slot; the claim is an atomic
+ * minimum, so the earliest arrival keeps the cell whatever order threads run in, and later ones count as n_dup.
+ * Arrival numbers continue from counters->n_arrived, so a further call in the same round (a retransmission
+ * attempt) never displaces an earlier packet.  recv_bitmap (W rows of row_words u32) is rewritten from slot_key.
+ *
+ * dblp_aggregate_reduce (Algorithm 2 "unreceived chunks remain 0-filled / reconstruct"; Algorithm 3 mean): for
+ * every element i of chunk c:  agg[i] = (+0.0f + x_0 + x_1 + ...) over the workers w = 0 .. W-1, in that order,
+ * whose cell (w, c) is claimed, x_w read from the claimed payload slot (bf16 widened exactly), plain fp32
+ * additions; with DBLP_MEAN the sum is divided by (float)W -- all workers, not the number that arrived.
+ * The destination is the plan's (tensor base + chunk offset), never the slot's position.  agg_out: N fp32.
+ *
+ * dblp_aggregate runs both.  slot_key, recv_bitmap and counters are in/out round state (dblp_round_reset). */
+int dblp_aggregate_book(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, uint64_t n_slots, const uint32_t* arrival,
+                        const uint64_t* n_arrived_dev, uint64_t arrival_cap, uint32_t round, uint32_t* recv_bitmap,
+                        uint64_t* slot_key, dblp_counters_t* counters, void* stream);
+int dblp_aggregate_reduce(const dblp_plan_t* plan, const void* payload_ring, const uint64_t* slot_key, float* agg_out,
+                          uint32_t flags, void* stream);
+int dblp_aggregate(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, const void* payload_ring, uint64_t n_slots,
+                   const uint32_t* arrival, const uint64_t* n_arrived_dev, uint64_t arrival_cap, uint32_t round,
+                   uint32_t* recv_bitmap, uint64_t* slot_key, dblp_counters_t* counters, float* agg_out,
+                   uint32_t flags, void* stream);
+
+/* Start of a round (Algorithm 2: bitmap <- 0): recv_bitmap <- 0, slot_key <- all-ones, counters <- 0. */
+int dblp_round_reset(const dblp_plan_t* plan, uint32_t* recv_bitmap, uint64_t* slot_key, dblp_counters_t* counters,
+                     void* stream);
+
+/* ---- check_bound (Section III-B: stop once missing / total <= p; Algorithm 2: stop signal or bitmap reply) ----
+ * For each worker w and bucket b: recv_cnt[w*B+b] = set bits of row w over the bucket's sequence range,
+ * missing_cnt = total - recv_cnt, ok = (missing * 10^6 <= bound_ppm * total) in 64-bit integers;
+ * *all_ok = 1 iff every ok is 1.  bound_ppm: HOST, n_bounds = 1 (one tolerance for all) or B (per bucket), in parts
+ * per million (Table I: 0.8 % = 8000).  Outputs: recv_cnt, missing_cnt u32[W*B], ok u8[W*B], all_ok u32[1]. */
+int dblp_check_bound(const dblp_plan_t* plan, const uint32_t* recv_bitmap, const uint32_t* bound_ppm,
+                     uint32_t n_bounds, uint32_t* recv_cnt, uint32_t* missing_cnt, uint8_t* ok, uint32_t* all_ok,
+                     void* stream);
+
+/* ---- phase-aware tolerance (HOST, pure) ----------------------------------------------------------------------
+ * dblp_clr: Eq. 1, |norm_prev - norm_curr| / norm_prev >= eta in fp64; norm_prev == 0 counts as critical.
+ * dblp_select_bound: Section IV-D / Algorithm 3: the first iteration uses P_low; at the start of an epoch the
+ * tolerance becomes P_high unless dblp_clr fires, then P_low; at any other iteration it stays current_ppm. */
+int dblp_clr(double norm_prev, double norm_curr, double eta);
+uint32_t dblp_select_bound(double norm_prev, double norm_curr, double eta, uint32_t p_low_ppm, uint32_t p_high_ppm,
+                           int at_epoch_start, int first_iteration, uint32_t current_ppm);
+
+/* ---- one whole round from HOST buffers --------------------------------------------------------------------------
+ * Copies each worker's gradient from host memory (pinned memory recommended) into dev->grads, runs
+ * round_reset, packetize, apply_loss, aggregate and check_bound, copies the aggregate, the counters and the bound
+ * outputs back to the host pointers and waits for the stream.  Every member of dblp_device_buffers_t is a device
+ * buffer the caller allocated with the sizes given; nothing is allocated here.  Host outputs may be NULL to skip. */
+typedef struct {
+    void* grads;               /* W * N elements of the plan's dtype, worker-major */
+    dblp_hdr_t* hdr_ring;      /* M headers */
+    void* payload_ring;        /* M * payload_bytes */
+    uint32_t* delivered_bits;  /* W * row_words */
+    uint32_t* arrival;         /* M */
+    uint64_t* n_arrived;       /* 1 */
+    uint32_t* recv_bitmap;     /* W * row_words */
+    uint64_t* slot_key;        /* W * C */
+    dblp_counters_t* counters; /* 1 */
+    float* agg;                /* N */
+    uint32_t* recv_cnt;        /* W * B */
+    uint32_t* missing_cnt;     /* W * B */
+    uint8_t* ok;               /* W * B */
+    uint32_t* all_ok;          /* 1 */
+    void* ws;
+    size_t ws_bytes;
+} dblp_device_buffers_t;
+
+int dblp_round_host(const dblp_plan_t* plan, const void* const* grads_host, const dblp_loss_model_t* model,
+                    uint64_t seed, uint32_t round, uint32_t bound_ppm, uint32_t flags,
+                    const dblp_device_buffers_t* dev, float* agg_host, dblp_counters_t* counters_host,
+                    uint32_t* recv_cnt_host, uint32_t* missing_cnt_host, uint8_t* ok_host, uint32_t* all_ok_host,
+                    void* stream);
+
+/* ---- diagnostics -----------------------------------------------------------------------------------------------*/
+const char* dblp_strerror(int status);
+const char* dblp_last_error(void);  /* HOST string, valid until the calling thread's next failing call */
+uint64_t dblp_launch_count(void);   /* kernels launched by this library since it was loaded */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DBLP_H */

@@ -125,7 +125,8 @@ int dblp_oracle_plan(const uint64_t* numel, uint32_t T, uint32_t elem_size, uint
  * Packetize (Algorithm 1, first step; Sections IV-A, IV-B).  For each worker,
  * tensor and chunk: copy the chunk into its payload slot and fill in the header.
  * Slot of packet (w, seq) is w*C + seq.  Bytes of a short chunk's slot past its
- * data length are written as zero.
+ * data length are written as zero.  With payload_ring == NULL only the headers
+ * are produced (they do not depend on the gradient values).
  * ------------------------------------------------------------------------- */
 int dblp_oracle_packetize(const uint64_t* numel, uint32_t T, uint32_t elem_size, uint32_t payload_bytes,
                           uint32_t W, const void* const* grads, uint32_t round,
@@ -138,7 +139,7 @@ int dblp_oracle_packetize(const uint64_t* numel, uint32_t T, uint32_t elem_size,
     if (rc) { free(base); free(cb); return rc; }
     uint64_t E = payload_bytes / elem_size, C = cb[T];
     for (uint32_t w = 0; w < W; ++w) {
-        const uint8_t* g = (const uint8_t*)grads[w];
+        const uint8_t* g = payload_ring ? (const uint8_t*)grads[w] : NULL;
         for (uint32_t t = 0; t < T; ++t) {
             uint64_t nchunks = (numel[t] + E - 1) / E;
             for (uint64_t j = 0; j < nchunks; ++j) {
@@ -154,6 +155,7 @@ int dblp_oracle_packetize(const uint64_t* numel, uint32_t T, uint32_t elem_size,
                 h->offset_elems = off;
                 h->worker = w;
                 h->reserved = 0;
+                if (!payload_ring) continue;
                 uint8_t* dst = payload_ring + slot * payload_bytes;
                 memcpy(dst, g + (base[t] + off) * elem_size, len * elem_size);
                 memset(dst + len * elem_size, 0, payload_bytes - len * elem_size);

@@ -115,6 +115,13 @@ class Plan:
                                            _p(hdr), _p(payload)), "packetize")
         return hdr, payload
 
+    def headers(self, rnd):
+        """Headers of all M packets without the payloads."""
+        hdr = np.zeros(self.M, HDR_DTYPE)
+        _check(lib().dblp_oracle_packetize(*self._args(), C.c_uint32(self.W), None, C.c_uint32(rnd), _p(hdr), None),
+               "packetize(headers)")
+        return hdr
+
     def header_at(self, w, seq, rnd):
         h = np.zeros(1, HDR_DTYPE)
         b = C.c_uint64()

@@ -1,0 +1,242 @@
+// dblp_aggregate: bookkeeping over the arrival list, then the masked fixed-order reduce
+// (Algorithm 2: integrity check, bitmap update, zero fill, reconstruction; Algorithm 3: mean over all workers;
+// Section III-A: packets of another round are dropped).
+//
+// k_book    one thread per arrival entry: 32-byte header read, checks against the plan's tables, one 64-bit atomic
+//           minimum on the claimed cell.  Integer atomics only, so every result is independent of thread order.
+// k_bitmap  warp ballot over the cells of a row -> one bitmap word per warp; also folds this call's arrival count
+//           into the counters (after every k_book thread has read the old value).
+// k_reduce  the bandwidth-bound kernel: one thread per (chunk, 16-byte vector).  It reads the W cell entries of its
+//           chunk, issues up to eight independent 128-bit streaming loads (one per worker that delivered), adds them
+//           in worker order into fp32 accumulators and writes the aggregate with 128-bit stores.  A worker whose
+//           packet was lost costs no payload traffic.
+#include "common.cuh"
+
+namespace dblp {
+
+constexpr int kBookThreads = 256;
+constexpr int kReduceThreads = 256;
+constexpr int kWorkerBatch = 8;
+
+// ------------------------------------------------------------------------------------------------ bookkeeping
+__global__ void __launch_bounds__(kBookThreads)
+k_book(const dblp_hdr_t* __restrict__ hdr_ring, uint64_t n_slots, const uint32_t* __restrict__ arrival,
+       const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap, uint32_t round,
+       unsigned long long* __restrict__ slot_key, dblp_counters_t* counters,
+       const uint64_t* __restrict__ numel, const uint32_t* __restrict__ chunkbase,
+       uint32_t T, uint32_t W, uint64_t C, uint32_t E, uint32_t es)
+{
+    const uint64_t n = min(*n_arrived_dev, arrival_cap);
+    const uint64_t a = (uint64_t)blockIdx.x * kBookThreads + threadIdx.x;
+    if ((uint64_t)blockIdx.x * kBookThreads >= n) return;          // whole block past the end
+    const uint64_t first_number = counters->n_arrived;             // arrival numbers continue across calls of a round
+    int accepted = 0, dup = 0, stale = 0, invalid = 0;
+    if (a < n) {
+        const uint32_t slot = __ldg(&arrival[a]);
+        bool valid = false;
+        uint4 h0 = make_uint4(0, 0, 0, 0), h1 = h0;
+        if (slot < n_slots) {
+            const uint4* hp = reinterpret_cast<const uint4*>(hdr_ring + slot);
+            h0 = __ldg(hp);       // seq, round, len_bytes, tensor_id
+            h1 = __ldg(hp + 1);   // offset lo, offset hi, worker, reserved
+            const uint64_t off = (uint64_t)h1.x | ((uint64_t)h1.y << 32);
+            if (h1.z < W && h0.w < T) {
+                const uint64_t nt = __ldg(&numel[h0.w]);
+                if (off < nt && off % E == 0) {
+                    const uint64_t len = min((uint64_t)E, nt - off);
+                    valid = (h0.z == len * es) && (h0.x == __ldg(&chunkbase[h0.w]) + off / E);
+                }
+            }
+        }
+        if (!valid) invalid = 1;
+        else if (h0.y != round) stale = 1;
+        else {
+            const unsigned long long key = ((first_number + a) << 32) | slot;
+            const unsigned long long old = atomicMin(&slot_key[(uint64_t)h1.z * C + h0.x], key);
+            if (old == kEmpty64) accepted = 1; else dup = 1;
+        }
+    }
+    const int n_acc = __syncthreads_count(accepted), n_dup = __syncthreads_count(dup);
+    const int n_stale = __syncthreads_count(stale), n_inv = __syncthreads_count(invalid);
+    if (threadIdx.x == 0) {
+        if (n_acc) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_accepted), (unsigned long long)n_acc);
+        if (n_dup) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_dup), (unsigned long long)n_dup);
+        if (n_stale) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_stale), (unsigned long long)n_stale);
+        if (n_inv) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_invalid), (unsigned long long)n_inv);
+    }
+}
+
+__global__ void __launch_bounds__(256)
+k_bitmap(const unsigned long long* __restrict__ slot_key, uint32_t* __restrict__ recv_bitmap, uint32_t W, uint64_t C,
+         uint64_t row_words, const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap, dblp_counters_t* counters)
+{
+    const uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;   // (row, word, lane)
+    const uint64_t row_bits = row_words * 32;
+    if (i == 0) {
+        const uint64_t total = counters->n_arrived + min(*n_arrived_dev, arrival_cap);
+        counters->n_arrived = total;
+        if (total > 0xFFFFFFFFull) counters->status |= 1u;
+    }
+    if (i >= row_bits * W) return;            // row_bits is a multiple of 32: whole warps leave together
+    const uint32_t w = (uint32_t)(i / row_bits);
+    const uint64_t c = i - (uint64_t)w * row_bits;
+    bool got = false;
+    if (c < C) got = reinterpret_cast<const uint2*>(slot_key)[(uint64_t)w * C + c].x != kEmpty32;
+    const uint32_t word = __ballot_sync(0xFFFFFFFFu, got);
+    if ((threadIdx.x & 31) == 0) recv_bitmap[(uint64_t)w * row_words + (c >> 5)] = word;
+}
+
+// ------------------------------------------------------------------------------------------------ reduce
+__device__ __forceinline__ uint4 ld_payload16(const uint8_t* p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ void st_agg16(float* p, float a, float b, float c, float d)
+{
+    asm volatile("st.global.cs.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
+template <int ES>
+__global__ void __launch_bounds__(kReduceThreads)
+k_reduce(const uint8_t* __restrict__ ring, const unsigned long long* __restrict__ slot_key,
+         const uint64_t* __restrict__ chunk_desc, float* __restrict__ agg, uint32_t W, uint32_t C, uint32_t P,
+         uint32_t VPC, int mean, float Wf)
+{
+    constexpr int VE = 16 / ES;            // elements per 16-byte vector: 4 fp32 or 8 bf16
+    const uint64_t i = (uint64_t)blockIdx.x * kReduceThreads + threadIdx.x;
+    if (i >= (uint64_t)C * VPC) return;
+    const uint32_t c = (uint32_t)(i / VPC), v = (uint32_t)(i - (uint64_t)c * VPC);
+    const uint64_t d = __ldg(&chunk_desc[c]);
+    const uint32_t len = (uint32_t)(d & 0xFFFFu), e0 = v * VE;
+    if (e0 >= len) return;
+
+    float acc[VE];
+#pragma unroll
+    for (int e = 0; e < VE; ++e) acc[e] = 0.0f;
+
+    const uint2* cell = reinterpret_cast<const uint2*>(slot_key) + c;   // low word = slot, all-ones = nothing arrived
+    for (uint32_t wb = 0; wb < W; wb += kWorkerBatch) {
+        uint32_t slot[kWorkerBatch];
+#pragma unroll
+        for (int k = 0; k < kWorkerBatch; ++k)
+            slot[k] = (wb + k < W) ? __ldg(&cell[(uint64_t)(wb + k) * C].x) : kEmpty32;
+        uint4 x[kWorkerBatch];
+#pragma unroll
+        for (int k = 0; k < kWorkerBatch; ++k)
+            if (slot[k] != kEmpty32) x[k] = ld_payload16(ring + (uint64_t)slot[k] * P + (uint64_t)v * 16);
+#pragma unroll
+        for (int k = 0; k < kWorkerBatch; ++k) {       // worker order: the additions are not reassociated
+            if (slot[k] == kEmpty32) continue;
+            if (ES == 4) {
+                acc[0] = __fadd_rn(acc[0], __uint_as_float(x[k].x));
+                acc[1] = __fadd_rn(acc[1], __uint_as_float(x[k].y));
+                acc[2] = __fadd_rn(acc[2], __uint_as_float(x[k].z));
+                acc[3] = __fadd_rn(acc[3], __uint_as_float(x[k].w));
+            } else {                                   // bf16 -> fp32 is a 16-bit shift
+                const uint32_t wd[4] = {x[k].x, x[k].y, x[k].z, x[k].w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    acc[2 * q] = __fadd_rn(acc[2 * q], __uint_as_float(wd[q] << 16));
+                    acc[2 * q + 1] = __fadd_rn(acc[2 * q + 1], __uint_as_float(wd[q] & 0xFFFF0000u));
+                }
+            }
+        }
+    }
+    if (mean) {
+#pragma unroll
+        for (int e = 0; e < VE; ++e) acc[e] = __fdiv_rn(acc[e], Wf);
+    }
+    float* out = agg + (d >> 16) + e0;
+    const uint32_t nv = min((uint32_t)VE, len - e0);
+    if (nv == VE && (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
+#pragma unroll
+        for (int q = 0; q < VE / 4; ++q) st_agg16(out + 4 * q, acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
+    } else {
+#pragma unroll
+        for (int e = 0; e < VE; ++e)
+            if (e < nv) out[e] = acc[e];
+    }
+}
+
+}  // namespace dblp
+
+using namespace dblp;
+
+extern "C" int dblp_aggregate_book(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, uint64_t n_slots,
+                                   const uint32_t* arrival, const uint64_t* n_arrived_dev, uint64_t arrival_cap,
+                                   uint32_t round, uint32_t* recv_bitmap, uint64_t* slot_key, dblp_counters_t* counters,
+                                   void* stream)
+{
+    DBLP_REQUIRE(plan && hdr_ring && arrival && n_arrived_dev && recv_bitmap && slot_key && counters, DBLP_EINVAL,
+                 "aggregate_book: null argument");
+    DBLP_REQUIRE(aligned16(hdr_ring), DBLP_EALIGN, "aggregate_book: header ring must be 16-byte aligned");
+    DBLP_REQUIRE(n_slots < 0xFFFFFFFFull, DBLP_ECAPACITY, "aggregate_book: ring has too many slots");
+    DBLP_REQUIRE(arrival_cap < (1ull << 32), DBLP_ECAPACITY, "aggregate_book: arrival list too long");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (arrival_cap > 0) {
+        const unsigned grid = (unsigned)((arrival_cap + kBookThreads - 1) / kBookThreads);
+        k_book<<<grid, kBookThreads, 0, s>>>(hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round,
+                                             reinterpret_cast<unsigned long long*>(slot_key), counters, plan->d_numel,
+                                             plan->d_chunkbase, plan->T, plan->W, plan->C, plan->E, plan->es);
+        DBLP_LAUNCHED();
+    }
+    const uint64_t cells = plan->row_words * 32 * plan->W;
+    k_bitmap<<<(unsigned)((cells + 255) / 256), 256, 0, s>>>(reinterpret_cast<const unsigned long long*>(slot_key),
+                                                           recv_bitmap, plan->W, plan->C, plan->row_words,
+                                                           n_arrived_dev, arrival_cap, counters);
+    DBLP_LAUNCHED();
+    return DBLP_OK;
+}
+
+extern "C" int dblp_aggregate_reduce(const dblp_plan_t* plan, const void* payload_ring, const uint64_t* slot_key,
+                                     float* agg_out, uint32_t flags, void* stream)
+{
+    DBLP_REQUIRE(plan && payload_ring && slot_key && agg_out, DBLP_EINVAL, "aggregate_reduce: null argument");
+    DBLP_REQUIRE(aligned16(payload_ring), DBLP_EALIGN, "aggregate_reduce: payload ring must be 16-byte aligned");
+    DBLP_REQUIRE((reinterpret_cast<uintptr_t>(agg_out) & 3u) == 0, DBLP_EALIGN, "aggregate_reduce: aggregate must be 4-byte aligned");
+    DBLP_REQUIRE(flags == DBLP_SUM || flags == DBLP_MEAN, DBLP_EINVAL, "aggregate_reduce: unknown flags %u", flags);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const uint64_t total = plan->C * plan->VPC;
+    const uint64_t grid = (total + kReduceThreads - 1) / kReduceThreads;
+    DBLP_REQUIRE(grid < (1ull << 31), DBLP_ECAPACITY, "aggregate_reduce: grid too large");
+    const int mean = flags == DBLP_MEAN;
+    if (plan->es == 4)
+        k_reduce<4><<<(unsigned)grid, kReduceThreads, 0, s>>>(static_cast<const uint8_t*>(payload_ring),
+            reinterpret_cast<const unsigned long long*>(slot_key), plan->d_chunk_desc, agg_out, plan->W,
+            (uint32_t)plan->C, plan->P, plan->VPC, mean, (float)plan->W);
+    else
+        k_reduce<2><<<(unsigned)grid, kReduceThreads, 0, s>>>(static_cast<const uint8_t*>(payload_ring),
+            reinterpret_cast<const unsigned long long*>(slot_key), plan->d_chunk_desc, agg_out, plan->W,
+            (uint32_t)plan->C, plan->P, plan->VPC, mean, (float)plan->W);
+    DBLP_LAUNCHED();
+    return DBLP_OK;
+}
+
+extern "C" int dblp_aggregate(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, const void* payload_ring,
+                              uint64_t n_slots, const uint32_t* arrival, const uint64_t* n_arrived_dev,
+                              uint64_t arrival_cap, uint32_t round, uint32_t* recv_bitmap, uint64_t* slot_key,
+                              dblp_counters_t* counters, float* agg_out, uint32_t flags, void* stream)
+{
+    DBLP_REQUIRE(payload_ring && agg_out, DBLP_EINVAL, "aggregate: null argument");
+    DBLP_REQUIRE(flags == DBLP_SUM || flags == DBLP_MEAN, DBLP_EINVAL, "aggregate: unknown flags %u", flags);
+    int rc = dblp_aggregate_book(plan, hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, recv_bitmap,
+                                 slot_key, counters, stream);
+    if (rc != DBLP_OK) return rc;
+    return dblp_aggregate_reduce(plan, payload_ring, slot_key, agg_out, flags, stream);
+}
+
+extern "C" int dblp_round_reset(const dblp_plan_t* plan, uint32_t* recv_bitmap, uint64_t* slot_key,
+                                dblp_counters_t* counters, void* stream)
+{
+    DBLP_REQUIRE(plan && recv_bitmap && slot_key && counters, DBLP_EINVAL, "round_reset: null argument");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    DBLP_CUDA(cudaMemsetAsync(recv_bitmap, 0, plan->row_words * plan->W * sizeof(uint32_t), s));
+    DBLP_CUDA(cudaMemsetAsync(slot_key, 0xFF, plan->M * sizeof(uint64_t), s));
+    DBLP_CUDA(cudaMemsetAsync(counters, 0, sizeof(dblp_counters_t), s));
+    return DBLP_OK;
+}

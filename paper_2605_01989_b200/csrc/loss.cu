@@ -1,0 +1,347 @@
+// dblp_apply_loss: the seeded loss process (delivered bitmap) and the permuted arrival list.
+// The paper injects loss without naming a generator (Section II-C "randomly zeroing out a fraction"; Section V-B
+// "manually injecting bursty packet loss"); the processes are defined in dblp.h, in integers, on Philox4x32-10 draws.
+//
+// Memoryless kinds (none / iid / microburst): one thread per packet, warp ballot -> one bitmap word per warp.
+// Gilbert-Elliott: the two-state chain is sequential by definition.  Each packet's transition is a function
+// {Good, Bad} -> {Good, Bad} (four possibilities, two bits); composition is associative, so the state at every packet
+// follows from a prefix "sum" of functions: one thread per bitmap word composes its 32 packets, a block scan and a
+// second small pass over the block totals give every word its entry state, and a third pass replays the 32 packets.
+// The start of a worker's row contributes a constant function (its drawn initial state), which resets the chain with
+// no special casing.  None of the passes waits on another block.
+// Arrival: pi(a) for a = 0 .. M-1 by a 4-round Feistel network with cycle walking; survivors are compacted in
+// order of a with ballot / popcount prefix sums over three passes.
+#include "common.cuh"
+
+namespace dblp {
+
+constexpr int kLossThreads = 256;
+constexpr int kGeThreads = 256;      // words per block in the chain passes
+constexpr int kScanThreads = 1024;   // single-block scans over block totals
+constexpr int kPermThreads = 1024;
+
+struct LossParams {
+    uint32_t kind;
+    uint64_t t_drop, t_gb, t_bg, t_init_bad, t_drop_good, t_drop_bad, window_len, t_drop_in, t_drop_out;
+};
+
+// ------------------------------------------------------------------------------------------------ memoryless kinds
+__global__ void __launch_bounds__(kLossThreads)
+k_loss_pointwise(LossParams m, DrawKey dk, uint32_t W, uint64_t C, uint64_t row_words, uint32_t* __restrict__ delivered)
+{
+    __shared__ uint64_t s_window_start;
+    if (m.kind == DBLP_LOSS_MICROBURST) {
+        if (threadIdx.x == 0) s_window_start = (uint64_t)draw(dk, 0, kStreamWindow).x % (C - m.window_len + 1);
+        __syncthreads();
+    }
+    const uint64_t i = (uint64_t)blockIdx.x * kLossThreads + threadIdx.x;   // (row, word, lane)
+    const uint64_t row_bits = row_words * 32;
+    if (i >= row_bits * W) return;
+    const uint32_t w = (uint32_t)(i / row_bits);
+    const uint64_t seq = i - (uint64_t)w * row_bits;
+    bool alive = false;
+    if (seq < C) {
+        uint64_t t = 0;
+        if (m.kind == DBLP_LOSS_IID) t = m.t_drop;
+        else if (m.kind == DBLP_LOSS_MICROBURST)
+            t = (seq >= s_window_start && seq < s_window_start + m.window_len) ? m.t_drop_in : m.t_drop_out;
+        const uint32_t u = draw(dk, (uint64_t)w * C + seq, kStreamPacket).x;
+        alive = !((uint64_t)u < t);
+    }
+    const uint32_t word = __ballot_sync(0xFFFFFFFFu, alive);
+    if ((threadIdx.x & 31) == 0) delivered[(uint64_t)w * row_words + (seq >> 5)] = word;
+}
+
+// ------------------------------------------------------------------------------------------------ Gilbert-Elliott
+// A function f on one bit is stored as f(0) | f(1) << 1.  State 0 = Good, 1 = Bad.
+__device__ __forceinline__ uint32_t fn_apply(uint32_t f, uint32_t x) { return (f >> x) & 1u; }
+__device__ __forceinline__ uint32_t fn_after(uint32_t later, uint32_t earlier)   // later o earlier
+{
+    return fn_apply(later, earlier & 1u) | (fn_apply(later, earlier >> 1) << 1);
+}
+constexpr uint32_t kFnIdentity = 2u;
+
+// Per word: bit masks over its (up to 32) packets of the four comparisons the chain needs, and the composed function
+// of the word including the row-start reset.
+struct GeWord {
+    uint32_t to_bad_if_good, stay_bad_if_bad, drop_if_good, drop_if_bad, valid;
+    uint32_t reset;   // kFnIdentity, or the constant function of the row's initial state
+    uint32_t fn;
+};
+
+__device__ __forceinline__ GeWord ge_word(const LossParams& m, const DrawKey& dk, uint64_t j, uint64_t C, uint64_t row_words)
+{
+    GeWord g{};
+    const uint32_t w = (uint32_t)(j / row_words);
+    const uint64_t k = j - (uint64_t)w * row_words;
+    g.reset = kFnIdentity;
+    if (k == 0) {
+        const uint32_t bad = (uint64_t)draw(dk, w, kStreamGeInit).x < m.t_init_bad;
+        g.reset = bad | (bad << 1);
+    }
+    uint32_t f = g.reset;
+    for (uint32_t b = 0; b < 32; ++b) {
+        const uint64_t seq = k * 32 + b;
+        if (seq >= C) break;
+        const uint4 u = draw(dk, (uint64_t)w * C + seq, kStreamPacket);
+        const uint32_t gb = (uint64_t)u.y < m.t_gb, bb = !((uint64_t)u.y < m.t_bg);
+        g.to_bad_if_good |= gb << b;
+        g.stay_bad_if_bad |= bb << b;
+        g.drop_if_good |= (uint32_t)((uint64_t)u.x < m.t_drop_good) << b;
+        g.drop_if_bad |= (uint32_t)((uint64_t)u.x < m.t_drop_bad) << b;
+        g.valid |= 1u << b;
+        f = fn_after(gb | (bb << 1), f);
+    }
+    g.fn = f;
+    return g;
+}
+
+// Exclusive scan of functions over a block (thread order = application order).  Returns the composition of all
+// earlier threads' functions; *block_total receives the whole block's.
+template <int THREADS>
+__device__ __forceinline__ uint32_t block_scan_fn(uint32_t f, uint32_t* block_total)
+{
+    __shared__ uint32_t s_warp[THREADS / 32];
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t inc = f;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= (uint32_t)d) inc = fn_after(inc, o);
+    }
+    if (lane == 31) s_warp[warp] = inc;
+    __syncthreads();
+    uint32_t before = kFnIdentity;                     // composition of the earlier warps
+    for (uint32_t k = 0; k < warp; ++k) before = fn_after(s_warp[k], before);
+    uint32_t exc = __shfl_up_sync(0xFFFFFFFFu, inc, 1);
+    if (lane == 0) exc = kFnIdentity;
+    exc = fn_after(exc, before);
+    if (threadIdx.x == THREADS - 1) *block_total = fn_after(f, exc);
+    return exc;
+}
+
+__global__ void __launch_bounds__(kGeThreads)
+k_ge_partial(LossParams m, DrawKey dk, uint32_t W, uint64_t C, uint64_t row_words, uint8_t* __restrict__ block_fn)
+{
+    __shared__ uint32_t s_total;
+    const uint64_t j = (uint64_t)blockIdx.x * kGeThreads + threadIdx.x;
+    uint32_t f = kFnIdentity;
+    if (j < row_words * W) f = ge_word(m, dk, j, C, row_words).fn;
+    block_scan_fn<kGeThreads>(f, &s_total);
+    __syncthreads();
+    if (threadIdx.x == 0) block_fn[blockIdx.x] = (uint8_t)s_total;
+}
+
+// One block: turns the per-block functions into the state with which each block is entered.
+__global__ void __launch_bounds__(kScanThreads)
+k_ge_block_states(const uint8_t* __restrict__ block_fn, uint8_t* __restrict__ block_state, uint32_t n_blocks)
+{
+    __shared__ uint32_t s_total;
+    const uint32_t per = (n_blocks + kScanThreads - 1) / kScanThreads;
+    const uint32_t lo = min(n_blocks, threadIdx.x * per), hi = min(n_blocks, lo + per);
+    uint32_t f = kFnIdentity;
+    for (uint32_t b = lo; b < hi; ++b) f = fn_after(block_fn[b], f);
+    uint32_t before = block_scan_fn<kScanThreads>(f, &s_total);
+    for (uint32_t b = lo; b < hi; ++b) {
+        block_state[b] = (uint8_t)fn_apply(before, 0);   // the value fed in is irrelevant: word 0 starts with a reset
+        before = fn_after(block_fn[b], before);
+    }
+}
+
+__global__ void __launch_bounds__(kGeThreads)
+k_ge_apply(LossParams m, DrawKey dk, uint32_t W, uint64_t C, uint64_t row_words,
+           const uint8_t* __restrict__ block_state, uint32_t* __restrict__ delivered)
+{
+    __shared__ uint32_t s_total;
+    const uint64_t j = (uint64_t)blockIdx.x * kGeThreads + threadIdx.x;
+    const bool live = j < row_words * W;
+    GeWord g{};
+    g.fn = kFnIdentity; g.reset = kFnIdentity;
+    if (live) g = ge_word(m, dk, j, C, row_words);
+    const uint32_t before = block_scan_fn<kGeThreads>(g.fn, &s_total);
+    if (!live) return;
+    uint32_t state = fn_apply(g.reset, fn_apply(before, block_state[blockIdx.x]));
+    uint32_t word = 0;
+    for (uint32_t b = 0; b < 32; ++b) {
+        if (!((g.valid >> b) & 1u)) break;
+        const uint32_t drop = ((state ? g.drop_if_bad : g.drop_if_good) >> b) & 1u;
+        word |= (drop ^ 1u) << b;
+        state = ((state ? g.stay_bad_if_bad : g.to_bad_if_good) >> b) & 1u;
+    }
+    delivered[j] = word;
+}
+
+// ------------------------------------------------------------------------------------------------ arrival order
+struct PermParams {
+    uint32_t half;   // bits per Feistel half
+    uint32_t mask;   // (1 << half) - 1
+    uint32_t M;
+};
+
+__device__ __forceinline__ uint32_t permute(const PermParams& pp, const DrawKey& dk, uint32_t a)
+{
+    uint32_t x = a;
+    do {   // a cycle of the permutation of [0, 2^b) that starts below M returns below M: the walk ends
+        uint32_t L = x >> pp.half, R = x & pp.mask;
+#pragma unroll
+        for (uint32_t r = 0; r < 4; ++r) {
+            const uint32_t F = philox4x32_10(make_uint4(R, r, kStreamPerm | dk.attempt8, dk.round), dk.key).x & pp.mask;
+            const uint32_t nl = R;
+            R = L ^ F;
+            L = nl;
+        }
+        x = (L << pp.half) | R;
+    } while (x >= pp.M);
+    return x;
+}
+
+__global__ void __launch_bounds__(kPermThreads)
+k_perm_flags(PermParams pp, DrawKey dk, uint64_t C, uint64_t row_words, const uint32_t* __restrict__ delivered,
+             uint32_t* __restrict__ perm_flag, uint32_t* __restrict__ block_count)
+{
+    const uint32_t a = blockIdx.x * kPermThreads + threadIdx.x;
+    int flag = 0;
+    if (a < pp.M) {
+        const uint32_t p = permute(pp, dk, a);
+        const uint32_t w = (uint32_t)(p / C);
+        const uint64_t seq = p - (uint64_t)w * C;
+        flag = (__ldg(&delivered[(uint64_t)w * row_words + (seq >> 5)]) >> (seq & 31)) & 1u;
+        perm_flag[a] = p | ((uint32_t)flag << 31);
+    }
+    const int n = __syncthreads_count(flag);
+    if (threadIdx.x == 0) block_count[blockIdx.x] = (uint32_t)n;
+}
+
+// One block: exclusive prefix sum of the per-block survivor counts (in place) and the total.
+__global__ void __launch_bounds__(kScanThreads)
+k_count_scan(uint32_t* __restrict__ block_count, uint32_t n_blocks, uint64_t* __restrict__ n_arrived)
+{
+    __shared__ uint32_t s_warp[kScanThreads / 32];
+    const uint32_t per = (n_blocks + kScanThreads - 1) / kScanThreads;
+    const uint32_t lo = min(n_blocks, threadIdx.x * per), hi = min(n_blocks, lo + per);
+    uint32_t sum = 0;
+    for (uint32_t b = lo; b < hi; ++b) sum += block_count[b];
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t inc = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= (uint32_t)d) inc += o;
+    }
+    if (lane == 31) s_warp[warp] = inc;
+    __syncthreads();
+    uint32_t before = 0;
+    for (uint32_t k = 0; k < warp; ++k) before += s_warp[k];
+    uint32_t run = before + inc - sum;
+    for (uint32_t b = lo; b < hi; ++b) {
+        const uint32_t n = block_count[b];
+        block_count[b] = run;
+        run += n;
+    }
+    if (threadIdx.x == kScanThreads - 1) *n_arrived = run;
+}
+
+__global__ void __launch_bounds__(kPermThreads)
+k_arrival_scatter(uint32_t M, const uint32_t* __restrict__ perm_flag, const uint32_t* __restrict__ block_offset,
+                  uint32_t* __restrict__ arrival)
+{
+    __shared__ uint32_t s_warp[kPermThreads / 32];
+    const uint32_t a = blockIdx.x * kPermThreads + threadIdx.x;
+    const uint32_t pf = a < M ? perm_flag[a] : 0u;
+    const bool flag = pf >> 31;
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t ballot = __ballot_sync(0xFFFFFFFFu, flag);
+    if (lane == 0) s_warp[warp] = __popc(ballot);
+    __syncthreads();
+    if (!flag) return;
+    uint32_t pos = block_offset[blockIdx.x] + __popc(ballot & ((1u << lane) - 1u));
+    for (uint32_t k = 0; k < warp; ++k) pos += s_warp[k];
+    arrival[pos] = pf & 0x7FFFFFFFu;
+}
+
+struct WorkspaceLayout {
+    size_t perm_flag, block_count, ge_fn, ge_state, total;
+    uint32_t n_perm_blocks, n_ge_blocks;
+};
+
+static WorkspaceLayout layout(const dblp_plan* p)
+{
+    WorkspaceLayout l{};
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    l.n_perm_blocks = (uint32_t)((p->M + kPermThreads - 1) / kPermThreads);
+    l.n_ge_blocks = (uint32_t)((p->row_words * p->W + kGeThreads - 1) / kGeThreads);
+    l.perm_flag = 0;
+    l.block_count = up(l.perm_flag + p->M * sizeof(uint32_t));
+    l.ge_fn = up(l.block_count + (size_t)l.n_perm_blocks * sizeof(uint32_t));
+    l.ge_state = up(l.ge_fn + l.n_ge_blocks);
+    l.total = up(l.ge_state + l.n_ge_blocks);
+    return l;
+}
+
+}  // namespace dblp
+
+using namespace dblp;
+
+extern "C" int dblp_workspace_bytes(const dblp_plan_t* plan, size_t* bytes)
+{
+    DBLP_REQUIRE(plan && bytes, DBLP_EINVAL, "workspace_bytes: null argument");
+    *bytes = layout(plan).total;
+    return DBLP_OK;
+}
+
+extern "C" int dblp_apply_loss(const dblp_plan_t* plan, const dblp_loss_model_t* model, uint64_t seed, uint32_t round,
+                               uint32_t attempt, uint32_t* delivered_bits, uint32_t* arrival, uint64_t* n_arrived_dev,
+                               void* ws, size_t ws_bytes, void* stream)
+{
+    DBLP_REQUIRE(plan && model && delivered_bits && arrival && n_arrived_dev && ws, DBLP_EINVAL, "apply_loss: null argument");
+    DBLP_REQUIRE(model->kind <= DBLP_LOSS_MICROBURST, DBLP_EINVAL, "apply_loss: unknown loss kind %u", model->kind);
+    DBLP_REQUIRE(attempt < (1u << 24), DBLP_ECAPACITY, "apply_loss: attempt must be below 2^24");
+    const WorkspaceLayout l = layout(plan);
+    DBLP_REQUIRE(ws_bytes >= l.total, DBLP_ECAPACITY, "apply_loss: workspace of %zu bytes, %zu needed", ws_bytes, l.total);
+    DBLP_REQUIRE((reinterpret_cast<uintptr_t>(ws) & 255u) == 0, DBLP_EALIGN, "apply_loss: workspace must be 256-byte aligned");
+    const uint64_t limit = 1ull << 32;
+    DBLP_REQUIRE(model->t_drop <= limit && model->t_gb <= limit && model->t_bg <= limit && model->t_init_bad <= limit &&
+                 model->t_drop_good <= limit && model->t_drop_bad <= limit && model->t_drop_in <= limit &&
+                 model->t_drop_out <= limit, DBLP_EINVAL, "apply_loss: thresholds must lie in [0, 2^32]");
+    if (model->kind == DBLP_LOSS_MICROBURST)
+        DBLP_REQUIRE(model->window_len <= plan->C, DBLP_EINVAL, "apply_loss: window longer than a worker's stream");
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint8_t* base = static_cast<uint8_t*>(ws);
+    uint32_t* perm_flag = reinterpret_cast<uint32_t*>(base + l.perm_flag);
+    uint32_t* block_count = reinterpret_cast<uint32_t*>(base + l.block_count);
+    uint8_t* ge_fn = base + l.ge_fn;
+    uint8_t* ge_state = base + l.ge_state;
+
+    LossParams m{model->kind, model->t_drop, model->t_gb, model->t_bg, model->t_init_bad, model->t_drop_good,
+                 model->t_drop_bad, model->window_len, model->t_drop_in, model->t_drop_out};
+    DrawKey dk{make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)), attempt << 8, round};
+
+    if (model->kind == DBLP_LOSS_GE) {
+        k_ge_partial<<<l.n_ge_blocks, kGeThreads, 0, s>>>(m, dk, plan->W, plan->C, plan->row_words, ge_fn);
+        DBLP_LAUNCHED();
+        k_ge_block_states<<<1, kScanThreads, 0, s>>>(ge_fn, ge_state, l.n_ge_blocks);
+        DBLP_LAUNCHED();
+        k_ge_apply<<<l.n_ge_blocks, kGeThreads, 0, s>>>(m, dk, plan->W, plan->C, plan->row_words, ge_state, delivered_bits);
+        DBLP_LAUNCHED();
+    } else {
+        const uint64_t threads = plan->row_words * 32 * plan->W;
+        k_loss_pointwise<<<(unsigned)((threads + kLossThreads - 1) / kLossThreads), kLossThreads, 0, s>>>(
+            m, dk, plan->W, plan->C, plan->row_words, delivered_bits);
+        DBLP_LAUNCHED();
+    }
+
+    PermParams pp{};
+    uint32_t bits = 2;
+    while (bits < 32 && (1ull << bits) < plan->M) bits += 2;
+    pp.half = bits / 2;
+    pp.mask = (1u << pp.half) - 1u;
+    pp.M = (uint32_t)plan->M;
+    k_perm_flags<<<l.n_perm_blocks, kPermThreads, 0, s>>>(pp, dk, plan->C, plan->row_words, delivered_bits, perm_flag, block_count);
+    DBLP_LAUNCHED();
+    k_count_scan<<<1, kScanThreads, 0, s>>>(block_count, l.n_perm_blocks, n_arrived_dev);
+    DBLP_LAUNCHED();
+    k_arrival_scatter<<<l.n_perm_blocks, kPermThreads, 0, s>>>(pp.M, perm_flag, block_count, arrival);
+    DBLP_LAUNCHED();
+    return DBLP_OK;
+}

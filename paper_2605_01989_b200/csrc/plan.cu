@@ -1,0 +1,204 @@
+// Plan creation (the constants of Section IV-A turned into device tables), host-side scalar rules (Eq. 1, the
+// tolerance schedule of Section IV-D / Algorithm 3) and diagnostics.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+
+#include <new>
+
+#include "common.cuh"
+
+namespace dblp {
+
+static thread_local char t_err[512] = "";
+std::atomic<uint64_t> g_launches{0};
+
+void set_error(const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(t_err, sizeof(t_err), fmt, ap);
+    va_end(ap);
+}
+
+static void free_tables(dblp_plan* p)
+{
+    cudaFree(p->d_numel);
+    cudaFree(p->d_base);
+    cudaFree(p->d_chunkbase);
+    cudaFree(p->d_chunk_desc);
+    cudaFree(p->d_chunk_tensor);
+    cudaFree(p->d_bucket_bounds);
+    cudaFree(p->d_bound_ppm);
+}
+
+template <typename T>
+static cudaError_t upload(T** dst, const std::vector<T>& src)
+{
+    cudaError_t e = cudaMalloc((void**)dst, src.size() * sizeof(T));
+    if (e != cudaSuccess) return e;
+    return cudaMemcpy(*dst, src.data(), src.size() * sizeof(T), cudaMemcpyHostToDevice);
+}
+
+}  // namespace dblp
+
+using namespace dblp;
+
+extern "C" int dblp_plan_create(const uint64_t* tensor_numel, uint32_t T, int dtype, uint32_t payload_bytes, uint32_t W,
+                                const uint64_t* bucket_seq_bounds, uint32_t B, dblp_plan_t** out)
+{
+    DBLP_REQUIRE(tensor_numel && out && T > 0 && W > 0 && B > 0, DBLP_EINVAL, "plan: null argument or zero count");
+    DBLP_REQUIRE(dtype == DBLP_F32 || dtype == DBLP_BF16, DBLP_EINVAL, "plan: unknown dtype %d", dtype);
+    DBLP_REQUIRE(payload_bytes >= 16 && payload_bytes <= 65536, DBLP_ECAPACITY, "plan: payload_bytes %u outside [16, 65536]",
+                 payload_bytes);
+    DBLP_REQUIRE(payload_bytes % 16 == 0, DBLP_EALIGN, "plan: payload_bytes %u is not a multiple of 16", payload_bytes);
+    DBLP_REQUIRE(bucket_seq_bounds || B == 1, DBLP_EINVAL, "plan: B = %u needs bucket_seq_bounds", B);
+
+    dblp_plan* p = new (std::nothrow) dblp_plan();
+    DBLP_REQUIRE(p, DBLP_EINVAL, "plan: out of host memory");
+    p->T = T; p->W = W; p->B = B; p->P = payload_bytes; p->dtype = dtype;
+    p->es = dtype == DBLP_F32 ? 4 : 2;
+    p->E = payload_bytes / p->es;
+    p->VE = 16 / p->es;
+    p->VPC = payload_bytes / 16;
+    p->d_numel = p->d_base = nullptr; p->d_chunk_desc = nullptr;
+    p->d_chunkbase = p->d_chunk_tensor = p->d_bucket_bounds = p->d_bound_ppm = nullptr;
+
+    uint64_t base = 0, c = 0;
+    p->h_numel.assign(tensor_numel, tensor_numel + T);
+    p->h_base.resize(T);
+    p->h_chunkbase.resize((size_t)T + 1);
+    for (uint32_t t = 0; t < T; ++t) {
+        if (tensor_numel[t] == 0) { delete p; DBLP_REQUIRE(false, DBLP_EINVAL, "plan: tensor %u has no elements", t); }
+        p->h_base[t] = base;
+        p->h_chunkbase[t] = (uint32_t)c;
+        base += tensor_numel[t];
+        c += (tensor_numel[t] + p->E - 1) / p->E;
+        if (base >= (1ull << 47) || c * W >= (1ull << 31)) {
+            delete p;
+            DBLP_REQUIRE(false, DBLP_ECAPACITY, "plan: W * C must stay below 2^31 packets and N below 2^47 elements");
+        }
+    }
+    p->h_chunkbase[T] = (uint32_t)c;
+    p->C = c; p->N = base; p->M = c * W; p->row_words = (c + 31) / 32;
+
+    std::vector<uint32_t> bounds((size_t)B + 1);
+    if (bucket_seq_bounds) {
+        bool ok = bucket_seq_bounds[0] == 0 && bucket_seq_bounds[B] == c;
+        for (uint32_t b = 0; b < B && ok; ++b) ok = bucket_seq_bounds[b] <= bucket_seq_bounds[b + 1];
+        if (!ok) { delete p; DBLP_REQUIRE(false, DBLP_EINVAL, "plan: bucket bounds must ascend from 0 to C = %llu", (unsigned long long)c); }
+        for (uint32_t b = 0; b <= B; ++b) bounds[b] = (uint32_t)bucket_seq_bounds[b];
+    } else {
+        bounds[0] = 0; bounds[1] = (uint32_t)c;
+    }
+
+    std::vector<uint64_t> desc(c);
+    std::vector<uint32_t> owner(c);
+    for (uint32_t t = 0; t < T; ++t) {
+        const uint64_t n = tensor_numel[t], nch = (n + p->E - 1) / p->E;
+        for (uint64_t j = 0; j < nch; ++j) {
+            const uint64_t off = j * p->E, len = n - off < p->E ? n - off : p->E;
+            desc[p->h_chunkbase[t] + j] = ((p->h_base[t] + off) << 16) | len;
+            owner[p->h_chunkbase[t] + j] = t;
+        }
+    }
+
+    cudaError_t e = cudaGetDevice(&p->device);
+    if (e == cudaSuccess) e = upload(&p->d_numel, p->h_numel);
+    if (e == cudaSuccess) e = upload(&p->d_base, p->h_base);
+    if (e == cudaSuccess) e = upload(&p->d_chunkbase, p->h_chunkbase);
+    if (e == cudaSuccess) e = upload(&p->d_chunk_desc, desc);
+    if (e == cudaSuccess) e = upload(&p->d_chunk_tensor, owner);
+    if (e == cudaSuccess) e = upload(&p->d_bucket_bounds, bounds);
+    if (e == cudaSuccess) e = cudaMalloc((void**)&p->d_bound_ppm, sizeof(uint32_t) * B);
+    if (e != cudaSuccess) {
+        set_error("plan: device table setup failed: %s", cudaGetErrorString(e));
+        free_tables(p);
+        delete p;
+        return DBLP_ECUDA;
+    }
+    *out = p;
+    return DBLP_OK;
+}
+
+extern "C" int dblp_plan_destroy(dblp_plan_t* plan)
+{
+    if (!plan) return DBLP_OK;
+    free_tables(plan);
+    delete plan;
+    return DBLP_OK;
+}
+
+extern "C" int dblp_plan_query(const dblp_plan_t* plan, uint64_t* C, uint64_t* N, uint64_t* M, uint64_t* row_words)
+{
+    DBLP_REQUIRE(plan, DBLP_EINVAL, "plan_query: null plan");
+    if (C) *C = plan->C;
+    if (N) *N = plan->N;
+    if (M) *M = plan->M;
+    if (row_words) *row_words = plan->row_words;
+    return DBLP_OK;
+}
+
+extern "C" int dblp_loss_model_from_rates(int kind, double mean_loss, double mean_burst_len, double window_frac,
+                                          double p_in, double p_out, uint64_t C, dblp_loss_model_t* out)
+{
+    DBLP_REQUIRE(out, DBLP_EINVAL, "loss_model_from_rates: null output");
+    auto thr = [](double p) -> uint64_t {
+        if (!(p > 0.0)) return 0;
+        if (p >= 1.0) return 1ull << 32;
+        return (uint64_t)floor(p * 4294967296.0);
+    };
+    *out = dblp_loss_model_t{};
+    out->kind = (uint32_t)kind;
+    switch (kind) {
+    case DBLP_LOSS_NONE: break;
+    case DBLP_LOSS_IID: out->t_drop = thr(mean_loss); break;
+    case DBLP_LOSS_GE: {
+        DBLP_REQUIRE(mean_burst_len >= 1.0 && mean_loss >= 0.0 && mean_loss <= 1.0, DBLP_EINVAL,
+                     "loss_model_from_rates: burst length must be >= 1 and loss within [0, 1]");
+        const double p_bg = 1.0 / mean_burst_len;
+        const double p_gb = mean_loss < 1.0 ? p_bg * mean_loss / (1.0 - mean_loss) : 1.0;
+        out->t_gb = thr(p_gb); out->t_bg = thr(p_bg); out->t_init_bad = thr(mean_loss);
+        out->t_drop_good = 0; out->t_drop_bad = 1ull << 32;
+        break;
+    }
+    case DBLP_LOSS_MICROBURST: {
+        uint64_t wl = (uint64_t)ceil(window_frac * (double)C);
+        out->window_len = wl > C ? C : wl;
+        out->t_drop_in = thr(p_in); out->t_drop_out = thr(p_out);
+        break;
+    }
+    default: DBLP_REQUIRE(false, DBLP_EINVAL, "loss_model_from_rates: unknown kind %d", kind);
+    }
+    return DBLP_OK;
+}
+
+extern "C" int dblp_clr(double norm_prev, double norm_curr, double eta)
+{
+    if (norm_prev == 0.0) return 1;
+    return fabs(norm_prev - norm_curr) / norm_prev >= eta ? 1 : 0;
+}
+
+extern "C" uint32_t dblp_select_bound(double norm_prev, double norm_curr, double eta, uint32_t p_low_ppm,
+                                      uint32_t p_high_ppm, int at_epoch_start, int first_iteration, uint32_t current_ppm)
+{
+    if (first_iteration) return p_low_ppm;
+    if (!at_epoch_start) return current_ppm;
+    return dblp_clr(norm_prev, norm_curr, eta) ? p_low_ppm : p_high_ppm;
+}
+
+extern "C" const char* dblp_strerror(int status)
+{
+    switch (status) {
+    case DBLP_OK: return "ok";
+    case DBLP_EINVAL: return "invalid argument";
+    case DBLP_EALIGN: return "misaligned pointer or size";
+    case DBLP_ECAPACITY: return "capacity or limit exceeded";
+    case DBLP_ECUDA: return "CUDA runtime error";
+    case DBLP_ETIMEOUT: return "timeout";
+    default: return "unknown status";
+    }
+}
+
+extern "C" const char* dblp_last_error(void) { return dblp::t_err; }
+extern "C" uint64_t dblp_launch_count(void) { return dblp::g_launches.load(std::memory_order_relaxed); }

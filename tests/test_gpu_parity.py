@@ -1,0 +1,252 @@
+"""GPU parity: the CUDA path, called through the C-ABI binding, against the CPU oracle on the same seeded inputs.
+Bar: bit-exact for headers, payloads, masks, arrival lists, bitmaps, slot tables, counters and bound decisions, and
+bit-exact for the fp32 aggregate (fixed worker order on both sides, bf16 widened exactly)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dblp_oracle as orc
+from paper_2605_01989_b200 import binding as dblp
+from paper_2605_01989_b200 import workloads as wl
+
+import harness as H
+
+pytestmark = pytest.mark.gpu
+
+RAGGED = [1000, 1, 352 * 40, 353, 7, 100003, 2, 352]          # sizes that are not multiples of the vector width
+ALIGNED = [1024, 4096 * 3, 64, 352 * 64, 8]
+
+
+def work(numel, dtype, P, W, loss, seed, bounds=(0, 8000, 50000, 408000)):
+    return wl.Workload("t", W, dtype, P, list(numel), 1e-3, loss, seed, bounds_ppm=bounds, round=seed + 3)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("P", [1408, 4096, 16])
+@pytest.mark.parametrize("loss", [wl.LossSpec("none"), wl.LossSpec("iid", 0.1), wl.LossSpec("ge", 0.1, 5.0),
+                                  wl.LossSpec("microburst", window_frac=0.2, p_in=0.5, p_out=0.01)],
+                         ids=["none", "iid", "ge", "mb"])
+def test_ragged_multi_tensor_round(dtype, P, loss):
+    numel = RAGGED if P != 16 else [37, 1, 8, 5, 4096]
+    H.full_round_parity(work(numel, dtype, P, 5, loss, 11))
+
+
+@pytest.mark.parametrize("W", [1, 2, 8, 9, 17, 32])
+def test_worker_counts(W):
+    H.full_round_parity(work(ALIGNED, "f32", 1024, W, wl.LossSpec("iid", 0.2), 5))
+
+
+def test_total_loss_and_zero_loss():
+    r = H.full_round_parity(work(RAGGED, "f32", 1408, 3, wl.LossSpec("iid", 1.0), 2))
+    assert r["n_arrived"] == 0
+    r = H.full_round_parity(work(RAGGED, "bf16", 1408, 3, wl.LossSpec("iid", 0.0), 2))
+    assert r["loss"] == 0.0
+
+
+def test_single_chunk_and_word_boundaries():
+    for n_chunks in (1, 31, 32, 33, 64, 65):
+        H.full_round_parity(work([256 * n_chunks], "f32", 1024, 2, wl.LossSpec("ge", 0.3, 3.0), n_chunks))
+
+
+def test_per_tensor_buckets_and_per_bucket_bounds():
+    w = work(RAGGED, "f32", 1408, 4, wl.LossSpec("iid", 0.05), 8)
+    op = orc.Plan(w.numel, 4, 1408, 4)
+    bb = [int(x) for x in op.chunkbase]
+    per_bucket = [0, 1000000, 50000, 20000, 0, 60000, 1000000, 0]
+    H.full_round_parity(w, bounds=[50000, per_bucket], bucket_bounds=bb)
+
+
+def test_config0_flat_fp32():
+    r = H.full_round_parity(wl.config(0))
+    assert 0.005 < r["loss"] < 0.015
+
+
+def test_config1_resnet50_shaped():
+    r = H.full_round_parity(wl.config(1), bounds=(24000, 8000, 0, 424000))
+    assert 0.004 < r["loss"] < 0.02
+
+
+def test_sweep_points_small():
+    pts = [wl.sweep_point(sz, W, P, loss, kind, seed)
+           for sz, W, P, loss, kind, seed in [(1 << 20, 2, 1024, 0.0, "iid", 10), (1 << 20, 32, 4096, 0.2, "ge", 11),
+                                              (1 << 22, 8, 1024, 0.05, "iid", 12), (1 << 22, 32, 1024, 0.01, "ge", 13),
+                                              (1 << 24, 2, 4096, 0.2, "iid", 14), (1 << 24, 8, 4096, 0.05, "ge", 10)]]
+    for p in pts:
+        H.full_round_parity(p, flags_list=(dblp.DBLP_SUM,))
+
+
+def test_stale_duplicate_and_invalid_packets_and_second_attempt():
+    w = work(RAGGED, "f32", 1408, 4, wl.LossSpec("iid", 0.3), 21)
+    rnd = w.round
+    grads = wl.make_grads(w, H.DEV)
+    host = H.to_host(grads, w.dtype)
+    op = orc.Plan(w.numel, 4, 1408, 4)
+    M, P = op.M, op.P
+    n_junk = 600
+    g = H.GpuRound(w, n_slots=M + n_junk, arrival_cap=2 * M)
+    gm, om = H.models_for(w, op.C)
+
+    # both sides packetize their own rings; the junk recipe below is applied to each side's ring separately
+    g.packetize(grads, rnd)
+    o_hdr, o_pay = op.packetize(host, rnd)
+    rng = np.random.default_rng(7)
+    src = rng.integers(0, M, n_junk)
+    kinds = rng.integers(0, 8, n_junk)
+
+    def add_junk(hdr, pay):
+        hdr = np.concatenate([hdr, hdr[src]])
+        pay = np.concatenate([pay.reshape(M, P), pay.reshape(M, P)[src]])
+        j = hdr[M:]
+        j["round"][kinds == 0] = rnd - 1
+        j["round"][kinds == 1] = rnd + 1
+        # kinds 2, 3: plain duplicates (payload of the copy is altered so that taking the wrong copy shows up)
+        pay[M:][np.isin(kinds, (2, 3))] ^= 0x5A
+        j["worker"][kinds == 4] = w.W + 3
+        j["tensor_id"][kinds == 5] = op.T
+        j["offset_elems"][kinds == 6] += 1
+        j["len_bytes"][kinds == 7] += 4
+        return hdr, pay.reshape(-1)
+
+    o_hdr2, o_pay2 = add_junk(o_hdr, o_pay)
+    g_hdr2, g_pay2 = add_junk(H.hdr_np(g.buf["hdr_ring"])[:M], g.buf["payload_ring"].cpu().numpy()[:M * P])
+    H.assert_bits_equal(g_hdr2, o_hdr2, "ring headers with junk")
+    g.buf["hdr_ring"].copy_(torch.from_numpy(g_hdr2.view(np.uint8).copy()))
+    g.buf["payload_ring"].copy_(torch.from_numpy(g_pay2.copy()))
+
+    # attempt 0: survivors of the loss process plus all junk slots plus an out-of-ring slot, shuffled
+    g.apply_loss(gm, w.seed, rnd)
+    o_del, _ = op.loss_mask(om, w.seed, rnd)
+    o_arr, o_n = op.arrival(o_del, w.seed, rnd)
+    H.assert_bits_equal(H.u32(g.buf["arrival"])[:o_n], o_arr[:o_n], "arrival list")
+    mixed = np.concatenate([o_arr[:o_n], np.arange(M, M + n_junk, dtype=np.uint32),
+                            np.array([M + n_junk, 0xFFFFFFFE], np.uint32)])
+    rng.shuffle(mixed)
+    g.buf["arrival"][:len(mixed)].copy_(torch.from_numpy(mixed.view(np.int32)))
+    g.buf["n_arrived"].fill_(len(mixed))
+    g.aggregate(rnd)
+    st = op.book(o_hdr2, mixed, len(mixed), rnd, op.new_state())
+    c = st["counters"].as_dict()
+    assert c["n_stale"] > 50 and c["n_dup"] > 50 and c["n_invalid"] > 100
+    H.compare_state(g, st, op)
+    H.assert_bits_equal(g.buf["agg"].cpu().numpy(), op.reduce(o_pay2, st), "aggregate with junk")
+
+    # attempt 1 of the same round: the sender re-sends what the bitmap says is missing; a new loss draw applies
+    g.apply_loss(gm, w.seed, rnd, attempt=1)
+    o_del1, _ = op.loss_mask(om, w.seed, rnd, attempt=1)
+    o_arr1, o_n1 = op.arrival(o_del1, w.seed, rnd, attempt=1)
+    H.assert_bits_equal(H.u32(g.buf["arrival"])[:o_n1], o_arr1[:o_n1], "arrival list, attempt 1")
+    g.aggregate(rnd, dblp.DBLP_MEAN)
+    st = op.book(o_hdr2, o_arr1, o_n1, rnd, st)
+    H.compare_state(g, st, op)
+    H.assert_bits_equal(g.buf["agg"].cpu().numpy(), op.reduce(o_pay2, st, mean=True), "aggregate after attempt 1")
+    assert st["counters"].as_dict()["n_dup"] > c["n_dup"]
+    H.compare_bound(g, op, st["bitmap"], 100000)
+    g.close()
+
+
+def test_physically_permuted_ring():
+    """Packets stored in the ring at their arrival position instead of slot w*C+seq: the receive path trusts headers
+    and the slot table only, so the aggregate must not change."""
+    w = work(ALIGNED + [100003], "bf16", 4096, 6, wl.LossSpec("ge", 0.1, 4.0), 31)
+    rnd = w.round
+    grads = wl.make_grads(w, H.DEV)
+    host = H.to_host(grads, w.dtype)
+    op = orc.Plan(w.numel, 2, 4096, 6)
+    gm, om = H.models_for(w, op.C)
+    g = H.GpuRound(w)
+    g.packetize(grads, rnd)
+    g.apply_loss(gm, w.seed, rnd)
+    n = g.n_arrived()
+    arr = g.buf["arrival"][:n].long()
+    # move payloads and headers of the survivors to ring positions 0..n-1 in arrival order (plumbing, torch indexing)
+    pay = g.buf["payload_ring"].view(op.M, op.P)
+    hdr = g.buf["hdr_ring"].view(op.M, 32)
+    pay[:n] = pay[arr].clone()
+    hdr[:n] = hdr[arr].clone()
+    pay[n:] = 0xEE
+    hdr[n:] = 0xEE                       # garbage in the rest of the ring must never be touched
+    g.buf["arrival"][:n] = torch.arange(n, dtype=torch.int32, device=H.DEV)
+    g.aggregate(rnd)
+    # oracle: its own round on the unpermuted ring -- the aggregate is defined by what arrived, not where it is stored
+    o_hdr, o_pay = op.packetize(host, rnd)
+    o_del, _ = op.loss_mask(om, w.seed, rnd)
+    o_arr, o_n = op.arrival(o_del, w.seed, rnd)
+    st = op.book(o_hdr, o_arr, o_n, rnd, op.new_state())
+    assert o_n == n
+    H.assert_bits_equal(g.buf["agg"].cpu().numpy(), op.reduce(o_pay, st), "aggregate from a permuted ring")
+    H.assert_bits_equal(H.u32(g.buf["recv_bitmap"]).reshape(op.W, op.row_words), st["bitmap"], "bitmap")
+    g.close()
+
+
+def test_round_host_entry_point_matches_the_oracle():
+    w = work(RAGGED, "f32", 1408, 3, wl.LossSpec("ge", 0.05, 6.0), 41)
+    op = orc.Plan(w.numel, 4, 1408, 3)
+    gm, om = H.models_for(w, op.C)
+    grads_host = [x.pin_memory() for x in wl.make_grads(w, "cpu")]
+    g = H.GpuRound(w)
+    grads_dev = torch.empty(w.W * w.N, dtype=torch.float32, device=H.DEV)
+    agg_host = torch.empty(w.N, dtype=torch.float32).pin_memory()
+    cnt_host = torch.zeros(6, dtype=torch.int64).pin_memory()
+    recv_host = torch.zeros(3, dtype=torch.int32).pin_memory()
+    miss_host = torch.zeros(3, dtype=torch.int32).pin_memory()
+    ok_host = torch.zeros(3, dtype=torch.uint8).pin_memory()
+    all_host = torch.zeros(1, dtype=torch.int32).pin_memory()
+    for rep in range(2):                       # second call reuses every buffer
+        dblp.dblp_round_host(g.plan, grads_host, gm, w.seed, w.round + rep, 60000, dblp.DBLP_MEAN, g.buf, grads_dev,
+                             agg_host, cnt_host, recv_host, miss_host, ok_host, all_host)
+        host = [x.numpy() for x in grads_host]
+        o_hdr, o_pay = op.packetize(host, w.round + rep)
+        o_del, _ = op.loss_mask(om, w.seed, w.round + rep)
+        o_arr, o_n = op.arrival(o_del, w.seed, w.round + rep)
+        st = op.book(o_hdr, o_arr, o_n, w.round + rep, op.new_state())
+        H.assert_bits_equal(agg_host.numpy(), op.reduce(o_pay, st, mean=True), "aggregate via round_host")
+        o = op.check_bound(st["bitmap"], 60000)
+        assert recv_host.numpy().view(np.uint32).tolist() == o[0][:, 0].tolist()
+        assert miss_host.numpy().view(np.uint32).tolist() == o[1][:, 0].tolist()
+        assert ok_host.numpy().tolist() == o[2][:, 0].tolist() and int(all_host[0]) == o[3]
+        assert dict(zip(dblp.COUNTER_FIELDS, cnt_host.tolist()[:5])) == st["counters"].as_dict()
+    g.close()
+
+
+def test_argument_errors_are_reported_not_faulted():
+    w = work(ALIGNED, "f32", 1024, 2, wl.LossSpec("iid", 0.1), 1)
+    g = H.GpuRound(w)
+    b = g.buf
+    with pytest.raises(dblp.DblpError) as e:
+        dblp.Plan([100], "f32", 1000, 2)                     # payload not a multiple of 16
+    assert e.value.status == -2
+    with pytest.raises(dblp.DblpError) as e:
+        dblp.Plan([100, 0], "f32", 1024, 2)                  # empty tensor
+    assert e.value.status == -1
+    with pytest.raises(dblp.DblpError) as e:
+        dblp.Plan([100], "f32", 1024, 2, bucket_seq_bounds=[0, 5])   # bounds must end at C
+    assert e.value.status == -1
+    with pytest.raises(dblp.DblpError) as e:                 # misaligned ring
+        dblp.dblp_packetize(g.plan, wl.make_grads(w, H.DEV), 1, b["hdr_ring"], b["payload_ring"][4:])
+    assert e.value.status == -2
+    with pytest.raises(dblp.DblpError) as e:                 # workspace too small
+        dblp.dblp_apply_loss(g.plan, dblp.loss_model("none"), 1, 1, 0, b["delivered_bits"], b["arrival"],
+                             b["n_arrived"], b["ws"][:1])
+    assert e.value.status == -3
+    with pytest.raises(dblp.DblpError) as e:                 # threshold above 2^32
+        dblp.dblp_apply_loss(g.plan, dblp.loss_model("iid", t_drop=(1 << 32) + 1), 1, 1, 0, b["delivered_bits"],
+                             b["arrival"], b["n_arrived"], b["ws"])
+    assert e.value.status == -1
+    with pytest.raises(dblp.DblpError) as e:
+        dblp.dblp_check_bound(g.plan, b["recv_bitmap"], [1, 2, 3], b["recv_cnt"], b["missing_cnt"], b["ok"], b["all_ok"])
+    assert e.value.status == -1
+    torch.cuda.synchronize()                                  # the context is still healthy
+    g.close()
+
+
+def test_library_counts_its_launches():
+    w = work(ALIGNED, "f32", 1024, 2, wl.LossSpec("ge", 0.1, 5.0), 1)
+    g = H.GpuRound(w)
+    gm, _ = H.models_for(w, g.plan.C)
+    n0 = dblp.dblp_launch_count()
+    g.packetize(wl.make_grads(w, H.DEV), 1)
+    g.apply_loss(gm, 1, 1)
+    g.aggregate(1)
+    g.check_bound(1000)
+    assert dblp.dblp_launch_count() - n0 == 1 + 6 + 3 + 2
+    g.close()
