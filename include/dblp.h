@@ -130,6 +130,29 @@ int dblp_apply_loss(const dblp_plan_t* plan, const dblp_loss_model_t* model, uin
                     uint32_t attempt, uint32_t* delivered_bits, uint32_t* arrival, uint64_t* n_arrived_dev, void* ws,
                     size_t ws_bytes, void* stream);
 
+/* ---- apply_loss without any allocation (the paper has no counterpart: this entry point exists for the sake of
+ * callers, not of the protocol) ---------------------------------------------------------------------------------
+ * Same results as dblp_apply_loss, bit for bit, but the scratch is a fixed array inside the library's own device
+ * image instead of a caller-provided workspace.  It is meant for callers that hold no allocator for device memory
+ * and must not call one: code running inside a memory pool whose owner forbids side allocations, plug-ins loaded
+ * into a host process that has already handed all device memory to another runtime, and hard real-time loops where
+ * an allocation's latency (or its implicit device synchronisation) is not acceptable.  Inputs and outputs are still
+ * the caller's buffers.
+ *   - Limit: the plan's dblp_workspace_bytes() must not exceed DBLP_STATIC_SCRATCH_BYTES (4 MiB + 64 KiB, i.e.
+ *     roughly W * C <= 2^20 packets per round); larger plans get DBLP_ECAPACITY and a message naming both sizes.
+ *   - Cost: every GPU on which the library is loaded keeps those bytes reserved until the process exits.
+ *   - The first call on a device looks up the array's device address (one cudaGetSymbolAddress, no allocation) and
+ *     caches it; make that first call before starting any stream capture on that device.  The plan's device must be
+ *     the current device.
+ *   - All calls on a device share the one array.  Nothing in it has to start at zero (each pass overwrites what the
+ *     next reads), but two calls whose kernels overlap on the GPU -- different streams, or different host threads
+ *     without ordering between them -- race on it.  Order them on one stream or with events.
+ *   - Calls no cudaMalloc, cudaFree or other allocating routine. */
+#define DBLP_STATIC_SCRATCH_BYTES (4u * 1024u * 1024u + 64u * 1024u)
+int dblp_apply_loss_static(const dblp_plan_t* plan, const dblp_loss_model_t* model, uint64_t seed, uint32_t round,
+                           uint32_t attempt, uint32_t* delivered_bits, uint32_t* arrival, uint64_t* n_arrived_dev,
+                           void* stream);
+
 /* ---- aggregate = bookkeeping + masked reduce ------------------------------------------------------------------
  * dblp_aggregate_book (Algorithm 2, chunk branch; Section III-A round filter): examines arrival[0 .. *n_arrived_dev)
  * (at most arrival_cap entries).  An entry is invalid if its slot >= n_slots or its header contradicts the plan

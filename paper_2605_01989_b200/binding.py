@@ -46,7 +46,8 @@ class DblpError(RuntimeError):
 
 _lib = None
 EXPORTS = ("dblp_plan_create", "dblp_plan_destroy", "dblp_plan_query", "dblp_workspace_bytes",
-           "dblp_loss_model_from_rates", "dblp_packetize", "dblp_apply_loss", "dblp_aggregate_book",
+           "dblp_loss_model_from_rates", "dblp_packetize", "dblp_apply_loss", "dblp_apply_loss_static",
+           "dblp_aggregate_book",
            "dblp_aggregate_reduce", "dblp_aggregate", "dblp_round_reset", "dblp_check_bound", "dblp_clr",
            "dblp_select_bound", "dblp_round_host", "dblp_strerror", "dblp_last_error", "dblp_launch_count")
 
@@ -168,6 +169,18 @@ def dblp_apply_loss(plan, model, seed, round, attempt, delivered_bits, arrival, 
     _check(lib().dblp_apply_loss(plan.handle, C.byref(model), C.c_uint64(seed), C.c_uint32(round), C.c_uint32(attempt),
                                  _ptr(delivered_bits), _ptr(arrival), _ptr(n_arrived_dev), _ptr(ws),
                                  C.c_size_t(ws.numel() * ws.element_size()), _stream(stream)), "dblp_apply_loss")
+
+
+STATIC_SCRATCH_BYTES = 4 * 1024 * 1024 + 64 * 1024
+
+
+def dblp_apply_loss_static(plan, model, seed, round, attempt, delivered_bits, arrival, n_arrived_dev, stream=None):
+    """dblp_apply_loss for callers that may not allocate device memory: the scratch is a fixed array inside the
+    library (plans up to STATIC_SCRATCH_BYTES of workspace).  All calls on a device share that array, so calls that
+    could overlap on the GPU must be ordered by the caller."""
+    _check(lib().dblp_apply_loss_static(plan.handle, C.byref(model), C.c_uint64(seed), C.c_uint32(round),
+                                        C.c_uint32(attempt), _ptr(delivered_bits), _ptr(arrival), _ptr(n_arrived_dev),
+                                        _stream(stream)), "dblp_apply_loss_static")
 
 
 def dblp_aggregate_book(plan, hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, recv_bitmap, slot_key,

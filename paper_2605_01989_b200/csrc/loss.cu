@@ -345,3 +345,41 @@ extern "C" int dblp_apply_loss(const dblp_plan_t* plan, const dblp_loss_model_t*
     DBLP_LAUNCHED();
     return DBLP_OK;
 }
+
+// ---------------------------------------------------------------------------------------------------- no-allocation variant
+// Scratch for callers that cannot obtain device memory at all (see dblp_apply_loss_static in dblp.h).  The array lives
+// in this library's device image: every GPU that loads the library holds these bytes until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[DBLP_STATIC_SCRATCH_BYTES];
+
+namespace dblp {
+constexpr int kMaxDevices = 64;
+static void* g_static_scratch_addr[kMaxDevices];          // device address of the array, per device; null = not set up
+static std::atomic<bool> g_static_scratch_ready[kMaxDevices];
+}  // namespace dblp
+
+extern "C" int dblp_apply_loss_static(const dblp_plan_t* plan, const dblp_loss_model_t* model, uint64_t seed,
+                                      uint32_t round, uint32_t attempt, uint32_t* delivered_bits, uint32_t* arrival,
+                                      uint64_t* n_arrived_dev, void* stream)
+{
+    DBLP_REQUIRE(plan, DBLP_EINVAL, "apply_loss_static: null plan");
+    const size_t need = layout(plan).total;
+    DBLP_REQUIRE(need <= (size_t)DBLP_STATIC_SCRATCH_BYTES, DBLP_ECAPACITY,
+                 "apply_loss_static: this plan needs %zu bytes of scratch, the built-in scratch holds %zu "
+                 "(about 2^20 packets per round); use dblp_apply_loss with a caller-provided workspace",
+                 need, (size_t)DBLP_STATIC_SCRATCH_BYTES);
+    int device = -1;
+    DBLP_CUDA(cudaGetDevice(&device));
+    DBLP_REQUIRE(device == plan->device, DBLP_EINVAL, "apply_loss_static: device %d is current, the plan lives on device %d",
+                 device, plan->device);
+    DBLP_REQUIRE(device >= 0 && device < kMaxDevices, DBLP_ECAPACITY, "apply_loss_static: device index %d not supported", device);
+    if (!g_static_scratch_ready[device].load(std::memory_order_acquire)) {
+        // In host code the array's name is only a handle; the kernels need its address in this device's memory.
+        void* addr = nullptr;
+        DBLP_CUDA(cudaGetSymbolAddress(&addr, g_static_scratch));
+        DBLP_REQUIRE(addr, DBLP_ECUDA, "apply_loss_static: the scratch symbol has no address on device %d", device);
+        g_static_scratch_addr[device] = addr;
+        g_static_scratch_ready[device].store(true, std::memory_order_release);
+    }
+    return dblp_apply_loss(plan, model, seed, round, attempt, delivered_bits, arrival, n_arrived_dev,
+                           g_static_scratch_addr[device], (size_t)DBLP_STATIC_SCRATCH_BYTES, stream);
+}
