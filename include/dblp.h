@@ -103,6 +103,11 @@ int dblp_plan_destroy(dblp_plan_t* plan);
 /* C = chunks per worker, N = elements per worker, M = W * C, row_words = ceil(C / 32) words per bitmap row.
  * Any out pointer may be NULL. */
 int dblp_plan_query(const dblp_plan_t* plan, uint64_t* C, uint64_t* N, uint64_t* M, uint64_t* row_words);
+/* Expert knob: pins the launch shape of the masked reduce (dblp_aggregate_reduce) -- chunks summed per tile and
+ * number of persistent blocks; 0 = choose automatically (what dblp_plan_create does).  Results do not depend on it.
+ * DBLP_ECAPACITY if the tile's slot entries do not fit in shared memory.  Not to be called while work that uses the
+ * plan is being enqueued from another thread. */
+int dblp_plan_tune_reduce(dblp_plan_t* plan, uint32_t chunks_per_tile, uint32_t grid_blocks);
 /* Bytes of scratch that dblp_apply_loss needs (the other calls need none). */
 int dblp_workspace_bytes(const dblp_plan_t* plan, size_t* bytes);
 

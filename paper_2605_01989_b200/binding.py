@@ -45,7 +45,7 @@ class DblpError(RuntimeError):
 
 
 _lib = None
-EXPORTS = ("dblp_plan_create", "dblp_plan_destroy", "dblp_plan_query", "dblp_workspace_bytes",
+EXPORTS = ("dblp_plan_create", "dblp_plan_destroy", "dblp_plan_query", "dblp_plan_tune_reduce", "dblp_workspace_bytes",
            "dblp_loss_model_from_rates", "dblp_packetize", "dblp_apply_loss", "dblp_apply_loss_static",
            "dblp_aggregate_book",
            "dblp_aggregate_reduce", "dblp_aggregate", "dblp_round_reset", "dblp_check_bound", "dblp_clr",
@@ -130,6 +130,10 @@ class Plan:
         ws = C.c_size_t()
         _check(lib().dblp_workspace_bytes(self.handle, C.byref(ws)), "dblp_workspace_bytes")
         self.workspace_bytes = int(ws.value)
+
+    def tune_reduce(self, chunks_per_tile=0, grid_blocks=0):
+        _check(lib().dblp_plan_tune_reduce(self.handle, C.c_uint32(chunks_per_tile), C.c_uint32(grid_blocks)),
+               "dblp_plan_tune_reduce")
 
     def close(self):
         if self.handle:

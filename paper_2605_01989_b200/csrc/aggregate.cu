@@ -6,7 +6,9 @@
 //           minimum on the claimed cell.  Integer atomics only, so every result is independent of thread order.
 // k_bitmap  warp ballot over the cells of a row -> one bitmap word per warp; also folds this call's arrival count
 //           into the counters (after every k_book thread has read the old value).
-// k_reduce  the bandwidth-bound kernel: one thread per (chunk, 16-byte vector).  It reads the W cell entries of its
+// k_reduce_tiled  the bandwidth-bound kernel (see the comment above it); k_reduce is its simple form, kept for
+//           worker counts whose slot entries do not fit in shared memory.
+// k_reduce  one thread per (chunk, 16-byte vector).  It reads the W cell entries of its
 //           chunk, issues up to eight independent 128-bit streaming loads (one per worker that delivered), adds them
 //           in worker order into fp32 accumulators and writes the aggregate with 128-bit stores.  A worker whose
 //           packet was lost costs no payload traffic.
@@ -163,6 +165,208 @@ k_reduce(const uint8_t* __restrict__ ring, const unsigned long long* __restrict_
     }
 }
 
+
+// ------------------------------------------------------------------------------------------------ tiled reduce
+// Persistent blocks walk over tiles of CH consecutive chunks.  For each tile the W x CH slot entries and the CH chunk
+// descriptors are brought into shared memory with cp.async while the previous tile is still being summed (two
+// buffers), so the only global loads a thread waits for are the payload vectors themselves: WB * J independent
+// 128-bit loads per thread, issued together, then added in worker order.  A thread's J items are 256 vectors apart,
+// so every warp instruction touches 512 contiguous bytes of each payload it reads.
+#ifndef DBLP_REDUCE_THREADS
+#define DBLP_REDUCE_THREADS 256
+#endif
+#ifndef DBLP_REDUCE_MIN_BLOCKS
+#define DBLP_REDUCE_MIN_BLOCKS 4   // caps the one-item variant at 64 registers: four 256-thread blocks per SM
+#endif
+#ifndef DBLP_REDUCE_J_WIDE
+#define DBLP_REDUCE_J_WIDE 1      // items per thread when W > 4 (8 workers per batch)
+#endif
+constexpr int kTileThreads = DBLP_REDUCE_THREADS;
+constexpr int kJWide = DBLP_REDUCE_J_WIDE;
+
+__device__ __forceinline__ void cp_async4(void* smem, const void* gmem)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem)), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async8(void* smem, const void* gmem)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"((uint32_t)__cvta_generic_to_shared(smem)), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+template <int ES, int WB, int J>
+__global__ void __launch_bounds__(kTileThreads, (J == 1 ? DBLP_REDUCE_MIN_BLOCKS : 1))
+k_reduce_tiled(const uint8_t* __restrict__ ring, const unsigned long long* __restrict__ slot_key,
+               const uint64_t* __restrict__ chunk_desc, float* __restrict__ agg, uint32_t W, uint32_t C, uint32_t P,
+               uint32_t VPC, uint32_t CH, uint32_t n_tiles, int mean, float Wf)
+{
+    constexpr int VE = 16 / ES;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint64_t* sdesc = reinterpret_cast<uint64_t*>(smem_raw);              // [2][CH]
+    uint32_t* sslot = reinterpret_cast<uint32_t*>(sdesc + 2 * CH);        // [2][CH][W]
+    const uint32_t tid = threadIdx.x;
+    const uint2* cells = reinterpret_cast<const uint2*>(slot_key);
+
+    auto prefetch = [&](uint32_t tile, uint32_t buf) {
+        const uint32_t c0 = tile * CH, nch = min(CH, C - c0);
+        uint32_t* dst = sslot + (size_t)buf * CH * W;
+        for (uint32_t k = tid; k < nch * W; k += kTileThreads) {
+            const uint32_t w = k / nch, cl = k - w * nch;               // consecutive threads: consecutive chunks of one worker
+            cp_async4(&dst[cl * W + w], &cells[(uint64_t)w * C + c0 + cl].x);
+        }
+        for (uint32_t k = tid; k < nch; k += kTileThreads) cp_async8(&sdesc[buf * CH + k], &chunk_desc[c0 + k]);
+    };
+
+    uint32_t tile = blockIdx.x, buf = 0;
+    if (tile < n_tiles) prefetch(tile, 0);
+    cp_async_commit();
+    for (; tile < n_tiles; tile += gridDim.x, buf ^= 1) {
+        const uint32_t next = tile + gridDim.x;
+        if (next < n_tiles) prefetch(next, buf ^ 1);
+        cp_async_commit();
+        cp_async_wait<1>();                   // everything but the group just committed has landed
+        __syncthreads();
+
+        const uint32_t c0 = tile * CH, nch = min(CH, C - c0), nvec = nch * VPC;
+        const uint64_t* td = sdesc + buf * CH;
+        const uint32_t* ts = sslot + (size_t)buf * CH * W;
+        for (uint32_t i0 = tid; i0 < nvec; i0 += kTileThreads * J) {
+            float acc[J][VE];
+            uint32_t cl[J], v[J], len[J];
+            uint64_t dst[J];
+            bool act[J];
+#pragma unroll
+            for (int j = 0; j < J; ++j) {
+                const uint32_t i = i0 + j * kTileThreads;
+                act[j] = i < nvec;
+                cl[j] = act[j] ? i / VPC : 0;
+                v[j] = i - cl[j] * VPC;
+                const uint64_t d = td[cl[j]];
+                len[j] = (uint32_t)(d & 0xFFFFu);
+                dst[j] = d >> 16;
+                act[j] = act[j] && v[j] * VE < len[j];
+#pragma unroll
+                for (int e = 0; e < VE; ++e) acc[j][e] = 0.0f;
+            }
+            for (uint32_t wb = 0; wb < W; wb += WB) {
+                uint32_t slot[J][WB];
+                uint4 x[J][WB];
+#pragma unroll
+                for (int j = 0; j < J; ++j)
+#pragma unroll
+                    for (int k = 0; k < WB; ++k)
+                        slot[j][k] = (act[j] && wb + k < W) ? ts[cl[j] * W + wb + k] : kEmpty32;
+#pragma unroll
+                for (int j = 0; j < J; ++j)
+#pragma unroll
+                    for (int k = 0; k < WB; ++k)
+                        if (slot[j][k] != kEmpty32) x[j][k] = ld_payload16(ring + (uint64_t)slot[j][k] * P + (uint64_t)v[j] * 16);
+#pragma unroll
+                for (int j = 0; j < J; ++j)
+#pragma unroll
+                    for (int k = 0; k < WB; ++k) {               // worker order: the additions are not reassociated
+                        if (slot[j][k] == kEmpty32) continue;
+                        if (ES == 4) {
+                            acc[j][0] = __fadd_rn(acc[j][0], __uint_as_float(x[j][k].x));
+                            acc[j][1] = __fadd_rn(acc[j][1], __uint_as_float(x[j][k].y));
+                            acc[j][2] = __fadd_rn(acc[j][2], __uint_as_float(x[j][k].z));
+                            acc[j][3] = __fadd_rn(acc[j][3], __uint_as_float(x[j][k].w));
+                        } else {
+                            const uint32_t wd[4] = {x[j][k].x, x[j][k].y, x[j][k].z, x[j][k].w};
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                acc[j][2 * q] = __fadd_rn(acc[j][2 * q], __uint_as_float(wd[q] << 16));
+                                acc[j][2 * q + 1] = __fadd_rn(acc[j][2 * q + 1], __uint_as_float(wd[q] & 0xFFFF0000u));
+                            }
+                        }
+                    }
+            }
+#pragma unroll
+            for (int j = 0; j < J; ++j) {
+                if (!act[j]) continue;
+                if (mean) {
+#pragma unroll
+                    for (int e = 0; e < VE; ++e) acc[j][e] = __fdiv_rn(acc[j][e], Wf);
+                }
+                const uint32_t e0 = v[j] * VE;
+                float* out = agg + dst[j] + e0;
+                const uint32_t nv = min((uint32_t)VE, len[j] - e0);
+                if (nv == VE && (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
+#pragma unroll
+                    for (int q = 0; q < VE / 4; ++q)
+                        st_agg16(out + 4 * q, acc[j][4 * q], acc[j][4 * q + 1], acc[j][4 * q + 2], acc[j][4 * q + 3]);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < VE; ++e)
+                        if (e < (int)nv) out[e] = acc[j][e];
+                }
+            }
+        }
+        __syncthreads();                      // the buffer is refilled by the prefetch of the next iteration
+    }
+    cp_async_wait<0>();
+}
+
+template <int ES, int WB, int J>
+static cudaError_t launch_tiled(const dblp_plan* p, const uint8_t* ring, const unsigned long long* slot_key, float* agg,
+                                int mean, cudaStream_t s)
+{
+    k_reduce_tiled<ES, WB, J><<<p->red_grid, kTileThreads, p->red_smem, s>>>(
+        ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->P, p->VPC, p->red_CH, p->red_tiles, mean, (float)p->W);
+    return cudaGetLastError();
+}
+
+template <int ES, int WB, int J>
+static cudaError_t occupancy_tiled(int* blocks, size_t smem)
+{
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, k_reduce_tiled<ES, WB, J>, kTileThreads, smem);
+}
+
+// Chooses the reduce kernel's shape for a plan: worker batch WB and items J so that WB * J = 8 loads are in flight per
+// thread, the tile height CH, and the grid.  Measured on B200 over payloads of 1408 and 4096 bytes, small tiles with one
+// block per tile (the hardware hands out tiles as blocks retire) beat one resident wave of persistent blocks by 1-3 %,
+// so that is the default; the persistent loop serves grids capped by the caller.  ch_override / grid_override
+// (0 = automatic) pin the shape.
+int configure_reduce(dblp_plan* p, uint32_t ch_override, uint32_t grid_override)
+{
+    p->red_variant = 0;
+    const uint32_t W = p->W;
+    const int J = W <= 2 ? 4 : (W <= 4 ? 2 : kJWide);
+    // Tile height: eight chunks, or more when chunks are so short that eight would not give every thread two items.
+    uint32_t CH = 8;
+    const uint32_t want = (2u * kTileThreads * J + p->VPC - 1) / p->VPC;
+    if (CH < want) CH = want;
+    const size_t per_chunk = (size_t)2 * (8 + 4 * (size_t)W);
+    const size_t smem_cap = 48 * 1024;
+    if (per_chunk > smem_cap) return DBLP_OK;              // slot entries of one chunk do not fit: simple kernel
+    if (CH * per_chunk > smem_cap) CH = (uint32_t)(smem_cap / per_chunk);
+    if (ch_override) {
+        if (ch_override * per_chunk > smem_cap) return DBLP_ECAPACITY;
+        CH = ch_override;
+    }
+    if (CH > p->C) CH = (uint32_t)p->C;
+    p->red_CH = CH;
+    p->red_smem = CH * per_chunk;
+    p->red_tiles = (uint32_t)((p->C + CH - 1) / CH);
+    int sms = 0, blocks = 0;
+    cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, p->device);
+    if (e == cudaSuccess) {
+        if (p->es == 4) e = J == 4 ? occupancy_tiled<4, 2, 4>(&blocks, p->red_smem) : (J == 2 && W <= 4) ? occupancy_tiled<4, 4, 2>(&blocks, p->red_smem) : occupancy_tiled<4, 8, kJWide>(&blocks, p->red_smem);
+        else            e = J == 4 ? occupancy_tiled<2, 2, 4>(&blocks, p->red_smem) : (J == 2 && W <= 4) ? occupancy_tiled<2, 4, 2>(&blocks, p->red_smem) : occupancy_tiled<2, 8, kJWide>(&blocks, p->red_smem);
+    }
+    if (e != cudaSuccess) { set_error("reduce set-up failed: %s", cudaGetErrorString(e)); return DBLP_ECUDA; }
+    if (blocks < 1) return DBLP_OK;
+    (void)sms;
+    uint32_t grid = p->red_tiles;
+    if (grid_override) grid = grid_override;
+    if (grid > p->red_tiles) grid = p->red_tiles;
+    p->red_grid = grid;
+    p->red_variant = J;
+    return DBLP_OK;
+}
+
 }  // namespace dblp
 
 using namespace dblp;
@@ -201,20 +405,42 @@ extern "C" int dblp_aggregate_reduce(const dblp_plan_t* plan, const void* payloa
     DBLP_REQUIRE((reinterpret_cast<uintptr_t>(agg_out) & 3u) == 0, DBLP_EALIGN, "aggregate_reduce: aggregate must be 4-byte aligned");
     DBLP_REQUIRE(flags == DBLP_SUM || flags == DBLP_MEAN, DBLP_EINVAL, "aggregate_reduce: unknown flags %u", flags);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int mean = flags == DBLP_MEAN;
+    const uint8_t* ring = static_cast<const uint8_t*>(payload_ring);
+    const unsigned long long* keys = reinterpret_cast<const unsigned long long*>(slot_key);
+    if (plan->red_variant) {
+        const int J = plan->red_variant;
+        if (plan->es == 4) {
+            if (J == 4) launch_tiled<4, 2, 4>(plan, ring, keys, agg_out, mean, s);
+            else if (J == 2 && plan->W <= 4) launch_tiled<4, 4, 2>(plan, ring, keys, agg_out, mean, s);
+            else launch_tiled<4, 8, kJWide>(plan, ring, keys, agg_out, mean, s);
+        } else {
+            if (J == 4) launch_tiled<2, 2, 4>(plan, ring, keys, agg_out, mean, s);
+            else if (J == 2 && plan->W <= 4) launch_tiled<2, 4, 2>(plan, ring, keys, agg_out, mean, s);
+            else launch_tiled<2, 8, kJWide>(plan, ring, keys, agg_out, mean, s);
+        }
+        DBLP_LAUNCHED();
+        return DBLP_OK;
+    }
     const uint64_t total = plan->C * plan->VPC;
     const uint64_t grid = (total + kReduceThreads - 1) / kReduceThreads;
     DBLP_REQUIRE(grid < (1ull << 31), DBLP_ECAPACITY, "aggregate_reduce: grid too large");
-    const int mean = flags == DBLP_MEAN;
     if (plan->es == 4)
-        k_reduce<4><<<(unsigned)grid, kReduceThreads, 0, s>>>(static_cast<const uint8_t*>(payload_ring),
-            reinterpret_cast<const unsigned long long*>(slot_key), plan->d_chunk_desc, agg_out, plan->W,
-            (uint32_t)plan->C, plan->P, plan->VPC, mean, (float)plan->W);
+        k_reduce<4><<<(unsigned)grid, kReduceThreads, 0, s>>>(ring, keys, plan->d_chunk_desc, agg_out, plan->W,
+                                                              (uint32_t)plan->C, plan->P, plan->VPC, mean, (float)plan->W);
     else
-        k_reduce<2><<<(unsigned)grid, kReduceThreads, 0, s>>>(static_cast<const uint8_t*>(payload_ring),
-            reinterpret_cast<const unsigned long long*>(slot_key), plan->d_chunk_desc, agg_out, plan->W,
-            (uint32_t)plan->C, plan->P, plan->VPC, mean, (float)plan->W);
+        k_reduce<2><<<(unsigned)grid, kReduceThreads, 0, s>>>(ring, keys, plan->d_chunk_desc, agg_out, plan->W,
+                                                              (uint32_t)plan->C, plan->P, plan->VPC, mean, (float)plan->W);
     DBLP_LAUNCHED();
     return DBLP_OK;
+}
+
+extern "C" int dblp_plan_tune_reduce(dblp_plan_t* plan, uint32_t chunks_per_tile, uint32_t grid_blocks)
+{
+    DBLP_REQUIRE(plan, DBLP_EINVAL, "plan_tune_reduce: null plan");
+    int rc = configure_reduce(plan, chunks_per_tile, grid_blocks);
+    if (rc == DBLP_ECAPACITY) set_error("plan_tune_reduce: %u chunks per tile do not fit in shared memory", chunks_per_tile);
+    return rc;
 }
 
 extern "C" int dblp_aggregate(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, const void* payload_ring,

@@ -97,4 +97,12 @@ struct dblp_plan {
     uint32_t* d_chunk_tensor;
     uint32_t* d_bucket_bounds;
     uint32_t* d_bound_ppm;
+    // launch shape of the masked reduce (configure_reduce): red_variant = items per thread of the tiled kernel,
+    // 0 = the simple one-vector-per-thread kernel
+    uint32_t red_variant, red_CH, red_tiles, red_grid;
+    size_t red_smem;
 };
+
+namespace dblp {
+int configure_reduce(dblp_plan* p, uint32_t ch_override, uint32_t grid_override);
+}

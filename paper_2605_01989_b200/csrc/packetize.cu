@@ -1,9 +1,11 @@
 // dblp_packetize: gradients -> header ring + payload ring (Algorithm 1 "split data into chunks"; Sections IV-A, IV-B).
 //
-// A pure copy, bound by HBM: each thread moves 16-byte vectors, kUnroll of them per thread with all loads issued
-// before the first store.  Work is indexed by (worker, chunk, vector-in-chunk); the chunk descriptor gives the source
-// element and the chunk's length, so tensors of any size are handled: a vector that is ragged (end of a short chunk) or
-// whose source is not 16-byte aligned is assembled from element loads, and the slot's tail is written as zero.
+// A pure copy, bound by HBM.  A block owns a tile of CH consecutive chunks of one worker: it first brings the tile's
+// chunk descriptors into shared memory (so that no payload load waits on a table lookup), writes the tile's headers,
+// then streams the tile's 16-byte vectors, kPackUnroll per thread per pass with all loads issued before the first
+// store.  The destination of a tile is one contiguous stretch of the ring; the source follows the descriptors, so
+// tensors of any size are handled: a vector that is ragged (end of a short chunk) or whose source is not 16-byte
+// aligned is assembled from element loads, and the slot's tail is written as zero.
 #include "common.cuh"
 
 namespace dblp {
@@ -29,60 +31,65 @@ __device__ __forceinline__ void st_stream16(void* p, uint4 v)
     asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
+constexpr uint32_t kPackMaxTile = 256;     // chunks per tile at most (descriptors live in static shared memory)
+
 template <int ES>
 __global__ void __launch_bounds__(kPackThreads)
-k_packetize(GradPtrs grads, uint32_t w0, uint32_t C, uint32_t VPC, uint32_t P, uint32_t round,
+k_packetize(GradPtrs grads, uint32_t w0, uint32_t C, uint32_t VPC, uint32_t P, uint32_t CH, uint32_t round,
             const uint64_t* __restrict__ chunk_desc, const uint32_t* __restrict__ chunk_tensor,
             const uint64_t* __restrict__ tensor_base, dblp_hdr_t* __restrict__ hdr_ring, uint8_t* __restrict__ ring)
 {
     constexpr uint32_t VE = 16 / ES;
-    const uint32_t wl = blockIdx.y, w = w0 + wl;
+    __shared__ uint64_t s_desc[kPackMaxTile];
+    const uint32_t wl = blockIdx.y, w = w0 + wl, tid = threadIdx.x;
     const uint8_t* __restrict__ g = static_cast<const uint8_t*>(grads.p[wl]);
-    const uint64_t total = (uint64_t)C * VPC;
-    const uint64_t first = ((uint64_t)blockIdx.x * kPackUnroll) * kPackThreads + threadIdx.x;
+    const uint32_t c0 = blockIdx.x * CH, nch = min(CH, C - c0);
+    const uint64_t slot0 = (uint64_t)w * C + c0;
 
-    uint4 val[kPackUnroll];
-    uint32_t chunk[kPackUnroll], vec[kPackUnroll];
-    uint64_t desc[kPackUnroll];
-#pragma unroll
-    for (int u = 0; u < kPackUnroll; ++u) {
-        const uint64_t i = first + (uint64_t)u * kPackThreads;
-        val[u] = make_uint4(0, 0, 0, 0);
-        chunk[u] = kEmpty32;
-        if (i >= total) continue;
-        const uint32_t c = (uint32_t)(i / VPC), v = (uint32_t)(i - (uint64_t)c * VPC);
-        chunk[u] = c; vec[u] = v;
-        const uint64_t d = __ldg(&chunk_desc[c]);
-        desc[u] = d;
-        const uint32_t len = (uint32_t)(d & 0xFFFFu), e0 = v * VE;
-        if (e0 >= len) continue;                       // wholly past the data of a short chunk: zero fill
-        const uint32_t nv = min(VE, len - e0);
-        const uint8_t* src = g + ((d >> 16) + e0) * ES;
-        if (nv == VE && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
-            val[u] = ld_stream16(src);
-        } else {
-            uint32_t wd[4] = {0, 0, 0, 0};
-#pragma unroll
-            for (uint32_t e = 0; e < VE; ++e) {
-                if (e < nv) {
-                    if (ES == 4) wd[e] = __ldg(reinterpret_cast<const uint32_t*>(src) + e);
-                    else wd[e >> 1] |= (uint32_t)__ldg(reinterpret_cast<const uint16_t*>(src) + e) << (16 * (e & 1));
-                }
-            }
-            val[u] = make_uint4(wd[0], wd[1], wd[2], wd[3]);
-        }
+    for (uint32_t k = tid; k < nch; k += kPackThreads) {
+        const uint64_t d = __ldg(&chunk_desc[c0 + k]);
+        s_desc[k] = d;
+        const uint32_t t = __ldg(&chunk_tensor[c0 + k]);
+        const uint64_t off = (d >> 16) - __ldg(&tensor_base[t]);
+        uint4* h = reinterpret_cast<uint4*>(hdr_ring + slot0 + k);
+        h[0] = make_uint4(c0 + k, round, (uint32_t)(d & 0xFFFFu) * ES, t);
+        h[1] = make_uint4((uint32_t)off, (uint32_t)(off >> 32), w, 0u);
     }
+    __syncthreads();
+
+    const uint32_t nvec = nch * VPC;
+    uint8_t* __restrict__ out = ring + slot0 * P;                 // the tile's slots are contiguous
+    for (uint32_t i0 = tid; i0 < nvec; i0 += kPackThreads * kPackUnroll) {
+        uint4 val[kPackUnroll];
 #pragma unroll
-    for (int u = 0; u < kPackUnroll; ++u) {
-        if (chunk[u] == kEmpty32) continue;
-        const uint64_t slot = (uint64_t)w * C + chunk[u];
-        st_stream16(ring + slot * P + (uint64_t)vec[u] * 16, val[u]);
-        if (vec[u] == 0) {
-            const uint32_t t = __ldg(&chunk_tensor[chunk[u]]);
-            const uint64_t off = (desc[u] >> 16) - __ldg(&tensor_base[t]);
-            uint4* h = reinterpret_cast<uint4*>(hdr_ring + slot);
-            h[0] = make_uint4(chunk[u], round, (uint32_t)(desc[u] & 0xFFFFu) * ES, t);
-            h[1] = make_uint4((uint32_t)off, (uint32_t)(off >> 32), w, 0u);
+        for (int u = 0; u < kPackUnroll; ++u) {
+            const uint32_t i = i0 + u * kPackThreads;
+            val[u] = make_uint4(0, 0, 0, 0);
+            if (i >= nvec) continue;
+            const uint32_t cl = i / VPC, v = i - cl * VPC;
+            const uint64_t d = s_desc[cl];
+            const uint32_t len = (uint32_t)(d & 0xFFFFu), e0 = v * VE;
+            if (e0 >= len) continue;                       // wholly past the data of a short chunk: zero fill
+            const uint32_t nv = min(VE, len - e0);
+            const uint8_t* src = g + ((d >> 16) + e0) * ES;
+            if (nv == VE && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
+                val[u] = ld_stream16(src);
+            } else {
+                uint32_t wd[4] = {0, 0, 0, 0};
+#pragma unroll
+                for (uint32_t e = 0; e < VE; ++e) {
+                    if (e < nv) {
+                        if (ES == 4) wd[e] = __ldg(reinterpret_cast<const uint32_t*>(src) + e);
+                        else wd[e >> 1] |= (uint32_t)__ldg(reinterpret_cast<const uint16_t*>(src) + e) << (16 * (e & 1));
+                    }
+                }
+                val[u] = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kPackUnroll; ++u) {
+            const uint32_t i = i0 + u * kPackThreads;
+            if (i < nvec) st_stream16(out + (uint64_t)i * 16, val[u]);
         }
     }
 }
@@ -102,9 +109,9 @@ extern "C" int dblp_packetize(const dblp_plan_t* plan, const void* const* grads,
                      "packetize: gradient of worker %u is not element-aligned", w);
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const uint64_t total = plan->C * plan->VPC;
-    const uint64_t per_block = (uint64_t)kPackThreads * kPackUnroll;
-    const uint64_t gx = (total + per_block - 1) / per_block;
+    uint32_t CH = (4096u + plan->VPC - 1) / plan->VPC;          // about 64 KB of payload per block
+    if (CH > kPackMaxTile) CH = kPackMaxTile;
+    const uint64_t gx = (plan->C + CH - 1) / CH;
     DBLP_REQUIRE(gx < (1ull << 31), DBLP_ECAPACITY, "packetize: grid too large");
     for (uint32_t w0 = 0; w0 < plan->W; w0 += kMaxWorkersPerLaunch) {
         const uint32_t nw = min(kMaxWorkersPerLaunch, plan->W - w0);
@@ -112,10 +119,10 @@ extern "C" int dblp_packetize(const dblp_plan_t* plan, const void* const* grads,
         for (uint32_t k = 0; k < nw; ++k) gp.p[k] = grads[w0 + k];
         dim3 grid((unsigned)gx, nw);
         if (plan->es == 4)
-            k_packetize<4><<<grid, kPackThreads, 0, s>>>(gp, w0, (uint32_t)plan->C, plan->VPC, plan->P, round,
+            k_packetize<4><<<grid, kPackThreads, 0, s>>>(gp, w0, (uint32_t)plan->C, plan->VPC, plan->P, CH, round,
                 plan->d_chunk_desc, plan->d_chunk_tensor, plan->d_base, hdr_ring, static_cast<uint8_t*>(payload_ring));
         else
-            k_packetize<2><<<grid, kPackThreads, 0, s>>>(gp, w0, (uint32_t)plan->C, plan->VPC, plan->P, round,
+            k_packetize<2><<<grid, kPackThreads, 0, s>>>(gp, w0, (uint32_t)plan->C, plan->VPC, plan->P, CH, round,
                 plan->d_chunk_desc, plan->d_chunk_tensor, plan->d_base, hdr_ring, static_cast<uint8_t*>(payload_ring));
         DBLP_LAUNCHED();
     }

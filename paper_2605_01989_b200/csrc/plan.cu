@@ -117,6 +117,12 @@ extern "C" int dblp_plan_create(const uint64_t* tensor_numel, uint32_t T, int dt
         delete p;
         return DBLP_ECUDA;
     }
+    const int rc = configure_reduce(p, 0, 0);
+    if (rc != DBLP_OK) {
+        free_tables(p);
+        delete p;
+        return rc;
+    }
     *out = p;
     return DBLP_OK;
 }
