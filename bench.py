@@ -134,7 +134,7 @@ def run_gpu(args):
     grads = wl.make_grads(work, dev)
     model = dblp.loss_model(work.loss.kind, **work.loss.thresholds(plan.C))
     bound = work.bounds_ppm[0]
-    count_vec = buf["recv_cnt"].view(torch.int32)
+    from paper_2605_01989_b200 import shard
 
     def step(rnd, ev=None):
         dblp.dblp_round_reset(plan, buf["recv_bitmap"], buf["slot_key"], buf["counters"])
@@ -152,8 +152,8 @@ def run_gpu(args):
         dblp.dblp_check_bound(plan, buf["recv_bitmap"], bound, buf["recv_cnt"], buf["missing_cnt"], buf["ok"],
                               buf["all_ok"])
         if ev: ev[5].record()
-        if dist is not None:
-            dist.all_reduce(count_vec)                 # the sharded path's one exchange: loss counts per worker
+        if dist is not None:                           # the sharded path's one exchange: loss counts per worker
+            shard.exchange_counts(buf["recv_cnt"], buf["missing_cnt"])
 
     for i in range(args.warmup):
         step(1 + i)

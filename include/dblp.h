@@ -198,6 +198,10 @@ int dblp_check_bound(const dblp_plan_t* plan, const uint32_t* recv_bitmap, const
                      uint32_t n_bounds, uint32_t* recv_cnt, uint32_t* missing_cnt, uint8_t* ok, uint32_t* all_ok,
                      void* stream);
 
+/* HOST, pure: the rule above for counts summed over several shards of one worker stream (each GPU of a sharded server
+ * counts its own chunk range): 1 iff missing * 10^6 <= bound_ppm * total.  Counts below 2^43 cannot overflow. */
+int dblp_bound_ok(uint64_t missing, uint64_t total, uint32_t bound_ppm);
+
 /* ---- phase-aware tolerance (HOST, pure) ----------------------------------------------------------------------
  * dblp_clr: Eq. 1, |norm_prev - norm_curr| / norm_prev >= eta in fp64; norm_prev == 0 counts as critical.
  * dblp_select_bound: Section IV-D / Algorithm 3: the first iteration uses P_low; at the start of an epoch the

@@ -48,7 +48,7 @@ _lib = None
 EXPORTS = ("dblp_plan_create", "dblp_plan_destroy", "dblp_plan_query", "dblp_plan_tune_reduce", "dblp_workspace_bytes",
            "dblp_loss_model_from_rates", "dblp_packetize", "dblp_apply_loss", "dblp_apply_loss_static",
            "dblp_aggregate_book",
-           "dblp_aggregate_reduce", "dblp_aggregate", "dblp_round_reset", "dblp_check_bound", "dblp_clr",
+           "dblp_aggregate_reduce", "dblp_aggregate", "dblp_round_reset", "dblp_check_bound", "dblp_bound_ok", "dblp_clr",
            "dblp_select_bound", "dblp_round_host", "dblp_strerror", "dblp_last_error", "dblp_launch_count")
 
 
@@ -217,6 +217,10 @@ def dblp_check_bound(plan, recv_bitmap, bound_ppm, recv_cnt, missing_cnt, ok, al
     arr = (C.c_uint32 * len(bounds))(*bounds)
     _check(lib().dblp_check_bound(plan.handle, _ptr(recv_bitmap), arr, C.c_uint32(len(bounds)), _ptr(recv_cnt),
                                   _ptr(missing_cnt), _ptr(ok), _ptr(all_ok), _stream(stream)), "dblp_check_bound")
+
+
+def dblp_bound_ok(missing, total, bound_ppm):
+    return bool(lib().dblp_bound_ok(C.c_uint64(missing), C.c_uint64(total), C.c_uint32(bound_ppm)))
 
 
 def dblp_clr(norm_prev, norm_curr, eta=0.5):

@@ -75,3 +75,9 @@ extern "C" int dblp_check_bound(const dblp_plan_t* plan, const uint32_t* recv_bi
     DBLP_LAUNCHED();
     return DBLP_OK;
 }
+
+// The same rule as k_bound's, on the host, for counts that were summed over several GPUs.
+extern "C" int dblp_bound_ok(uint64_t missing, uint64_t total, uint32_t bound_ppm)
+{
+    return missing * 1000000ull <= (uint64_t)bound_ppm * total ? 1 : 0;
+}
