@@ -5,20 +5,25 @@
 // Memoryless kinds (none / iid / microburst): one thread per packet, warp ballot -> one bitmap word per warp.
 // Gilbert-Elliott: the two-state chain is sequential by definition.  Each packet's transition is a function
 // {Good, Bad} -> {Good, Bad} (four possibilities, two bits); composition is associative, so the state at every packet
-// follows from a prefix "sum" of functions: one thread per bitmap word composes its 32 packets, a block scan and a
-// second small pass over the block totals give every word its entry state, and a third pass replays the 32 packets.
+// follows from a prefix "sum" of functions: a warp draws the 32 packets of a bitmap word in parallel and scans their
+// functions with shuffles, a block combines its warps, a second small pass over the block totals gives every block
+// its entry state, and a third pass judges every packet in its now known state (ballot -> bitmap word).
 // The start of a worker's row contributes a constant function (its drawn initial state), which resets the chain with
 // no special casing.  None of the passes waits on another block.
-// Arrival: pi(a) for a = 0 .. M-1 by a 4-round Feistel network with cycle walking; survivors are compacted in
+// Arrival: pi(a) for a = 0 .. M-1 by a 4-round Feistel network with cycle walking (each thread walks four
+// consecutive a one after the other, which evens out the walk lengths across a warp); survivors are compacted in
 // order of a with ballot / popcount prefix sums over three passes.
 #include "common.cuh"
 
 namespace dblp {
 
 constexpr int kLossThreads = 256;
-constexpr int kGeThreads = 256;      // words per block in the chain passes
+constexpr int kGeThreads = 256;
+constexpr int kGeWordsPerWarp = 4;
+constexpr int kGeWordsPerBlock = kGeThreads / 32 * kGeWordsPerWarp;   // bitmap words one block of the chain passes covers
 constexpr int kScanThreads = 1024;   // single-block scans over block totals
-constexpr int kPermThreads = 1024;
+constexpr int kPermThreads = 1024;   // arrival positions per block of the compaction passes
+constexpr int kPermWalkers = 256;    // threads of k_perm_flags; each walks kPermThreads / kPermWalkers positions
 
 struct LossParams {
     uint32_t kind;
@@ -61,47 +66,92 @@ __device__ __forceinline__ uint32_t fn_after(uint32_t later, uint32_t earlier)  
 }
 constexpr uint32_t kFnIdentity = 2u;
 
-// Per word: bit masks over its (up to 32) packets of the four comparisons the chain needs, and the composed function
-// of the word including the row-start reset.
-struct GeWord {
-    uint32_t to_bad_if_good, stay_bad_if_bad, drop_if_good, drop_if_bad, valid;
-    uint32_t reset;   // kFnIdentity, or the constant function of the row's initial state
-    uint32_t fn;
+// One bitmap word (row w, word k) handled by a whole warp: lane b owns packet k*32+b.
+struct GeLane {
+    uint32_t before;     // composition of the word's packets that precede this lane's (identity for lane 0)
+    uint32_t word_fn;    // composition of all the word's packets (uniform across the warp)
+    uint32_t reset;      // kFnIdentity, or the constant function of the row's initial state (first word of a row)
+    bool valid, drop_if_good, drop_if_bad;
 };
 
-__device__ __forceinline__ GeWord ge_word(const LossParams& m, const DrawKey& dk, uint64_t j, uint64_t C, uint64_t row_words)
+__device__ __forceinline__ GeLane ge_word(const LossParams& m, const DrawKey& dk, uint64_t j, uint64_t C, uint64_t row_words)
 {
-    GeWord g{};
+    GeLane g;
+    const uint32_t lane = threadIdx.x & 31;
     const uint32_t w = (uint32_t)(j / row_words);
     const uint64_t k = j - (uint64_t)w * row_words;
+    const uint64_t seq = k * 32 + lane;
+    g.valid = seq < C;
+    uint32_t fn = kFnIdentity;          // padding bits past the end of the row leave the state alone
+    g.drop_if_good = g.drop_if_bad = false;
+    if (g.valid) {
+        const uint4 u = draw(dk, (uint64_t)w * C + seq, kStreamPacket);
+        const uint32_t to_bad = (uint64_t)u.y < m.t_gb, stay_bad = !((uint64_t)u.y < m.t_bg);
+        fn = to_bad | (stay_bad << 1);
+        g.drop_if_good = (uint64_t)u.x < m.t_drop_good;
+        g.drop_if_bad = (uint64_t)u.x < m.t_drop_bad;
+    }
+    uint32_t inc = fn;                  // inclusive scan over the lanes: lower lanes are applied first
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+        if (lane >= (uint32_t)d) inc = fn_after(inc, o);
+    }
+    g.before = __shfl_up_sync(0xFFFFFFFFu, inc, 1);
+    if (lane == 0) g.before = kFnIdentity;
+    g.word_fn = __shfl_sync(0xFFFFFFFFu, inc, 31);
     g.reset = kFnIdentity;
     if (k == 0) {
         const uint32_t bad = (uint64_t)draw(dk, w, kStreamGeInit).x < m.t_init_bad;
         g.reset = bad | (bad << 1);
     }
-    uint32_t f = g.reset;
-    for (uint32_t b = 0; b < 32; ++b) {
-        const uint64_t seq = k * 32 + b;
-        if (seq >= C) break;
-        const uint4 u = draw(dk, (uint64_t)w * C + seq, kStreamPacket);
-        const uint32_t gb = (uint64_t)u.y < m.t_gb, bb = !((uint64_t)u.y < m.t_bg);
-        g.to_bad_if_good |= gb << b;
-        g.stay_bad_if_bad |= bb << b;
-        g.drop_if_good |= (uint32_t)((uint64_t)u.x < m.t_drop_good) << b;
-        g.drop_if_bad |= (uint32_t)((uint64_t)u.x < m.t_drop_bad) << b;
-        g.valid |= 1u << b;
-        f = fn_after(gb | (bb << 1), f);
-    }
-    g.fn = f;
     return g;
 }
 
-// Exclusive scan of functions over a block (thread order = application order).  Returns the composition of all
-// earlier threads' functions; *block_total receives the whole block's.
-template <int THREADS>
-__device__ __forceinline__ uint32_t block_scan_fn(uint32_t f, uint32_t* block_total)
+// Composition of the functions of the block's warps that come before this warp; *block_total receives all of them.
+// warp_fn is uniform within each warp.
+__device__ __forceinline__ uint32_t ge_block_prefix(uint32_t warp_fn, uint32_t* block_total)
 {
-    __shared__ uint32_t s_warp[THREADS / 32];
+    __shared__ uint32_t s_warp[kGeThreads / 32];
+    const uint32_t warp = threadIdx.x >> 5;
+    if ((threadIdx.x & 31) == 0) s_warp[warp] = warp_fn;
+    __syncthreads();
+    uint32_t before = kFnIdentity, all = kFnIdentity;
+    for (uint32_t k = 0; k < kGeThreads / 32; ++k) {
+        if (k == warp) before = all;
+        all = fn_after(s_warp[k], all);
+    }
+    *block_total = all;
+    return before;
+}
+
+__global__ void __launch_bounds__(kGeThreads)
+k_ge_partial(LossParams m, DrawKey dk, uint32_t W, uint64_t C, uint64_t row_words, uint8_t* __restrict__ block_fn)
+{
+    const uint64_t n_words = row_words * W;
+    const uint64_t j0 = (uint64_t)blockIdx.x * kGeWordsPerBlock + (threadIdx.x >> 5) * kGeWordsPerWarp;
+    uint32_t f = kFnIdentity;
+    for (int q = 0; q < kGeWordsPerWarp; ++q) {
+        if (j0 + q < n_words) {
+            const GeLane g = ge_word(m, dk, j0 + q, C, row_words);
+            f = fn_after(g.word_fn, fn_after(g.reset, f));
+        }
+    }
+    uint32_t total;
+    ge_block_prefix(f, &total);
+    if (threadIdx.x == 0) block_fn[blockIdx.x] = (uint8_t)total;
+}
+
+// One block: turns the per-block functions into the state with which each block is entered.
+__global__ void __launch_bounds__(kScanThreads)
+k_ge_block_states(const uint8_t* __restrict__ block_fn, uint8_t* __restrict__ block_state, uint32_t n_blocks)
+{
+    __shared__ uint32_t s_warp[kScanThreads / 32];
+    const uint32_t per = (n_blocks + kScanThreads - 1) / kScanThreads;
+    const uint32_t lo = min(n_blocks, threadIdx.x * per), hi = min(n_blocks, lo + per);
+    uint32_t f = kFnIdentity;
+    for (uint32_t b = lo; b < hi; ++b) f = fn_after(block_fn[b], f);
+    // exclusive scan of f over the block's threads (thread order = application order)
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t inc = f;
 #pragma unroll
@@ -111,37 +161,11 @@ __device__ __forceinline__ uint32_t block_scan_fn(uint32_t f, uint32_t* block_to
     }
     if (lane == 31) s_warp[warp] = inc;
     __syncthreads();
-    uint32_t before = kFnIdentity;                     // composition of the earlier warps
+    uint32_t before = kFnIdentity;
     for (uint32_t k = 0; k < warp; ++k) before = fn_after(s_warp[k], before);
     uint32_t exc = __shfl_up_sync(0xFFFFFFFFu, inc, 1);
     if (lane == 0) exc = kFnIdentity;
-    exc = fn_after(exc, before);
-    if (threadIdx.x == THREADS - 1) *block_total = fn_after(f, exc);
-    return exc;
-}
-
-__global__ void __launch_bounds__(kGeThreads)
-k_ge_partial(LossParams m, DrawKey dk, uint32_t W, uint64_t C, uint64_t row_words, uint8_t* __restrict__ block_fn)
-{
-    __shared__ uint32_t s_total;
-    const uint64_t j = (uint64_t)blockIdx.x * kGeThreads + threadIdx.x;
-    uint32_t f = kFnIdentity;
-    if (j < row_words * W) f = ge_word(m, dk, j, C, row_words).fn;
-    block_scan_fn<kGeThreads>(f, &s_total);
-    __syncthreads();
-    if (threadIdx.x == 0) block_fn[blockIdx.x] = (uint8_t)s_total;
-}
-
-// One block: turns the per-block functions into the state with which each block is entered.
-__global__ void __launch_bounds__(kScanThreads)
-k_ge_block_states(const uint8_t* __restrict__ block_fn, uint8_t* __restrict__ block_state, uint32_t n_blocks)
-{
-    __shared__ uint32_t s_total;
-    const uint32_t per = (n_blocks + kScanThreads - 1) / kScanThreads;
-    const uint32_t lo = min(n_blocks, threadIdx.x * per), hi = min(n_blocks, lo + per);
-    uint32_t f = kFnIdentity;
-    for (uint32_t b = lo; b < hi; ++b) f = fn_after(block_fn[b], f);
-    uint32_t before = block_scan_fn<kScanThreads>(f, &s_total);
+    before = fn_after(exc, before);
     for (uint32_t b = lo; b < hi; ++b) {
         block_state[b] = (uint8_t)fn_apply(before, 0);   // the value fed in is irrelevant: word 0 starts with a reset
         before = fn_after(block_fn[b], before);
@@ -152,23 +176,31 @@ __global__ void __launch_bounds__(kGeThreads)
 k_ge_apply(LossParams m, DrawKey dk, uint32_t W, uint64_t C, uint64_t row_words,
            const uint8_t* __restrict__ block_state, uint32_t* __restrict__ delivered)
 {
-    __shared__ uint32_t s_total;
-    const uint64_t j = (uint64_t)blockIdx.x * kGeThreads + threadIdx.x;
-    const bool live = j < row_words * W;
-    GeWord g{};
-    g.fn = kFnIdentity; g.reset = kFnIdentity;
-    if (live) g = ge_word(m, dk, j, C, row_words);
-    const uint32_t before = block_scan_fn<kGeThreads>(g.fn, &s_total);
-    if (!live) return;
-    uint32_t state = fn_apply(g.reset, fn_apply(before, block_state[blockIdx.x]));
-    uint32_t word = 0;
-    for (uint32_t b = 0; b < 32; ++b) {
-        if (!((g.valid >> b) & 1u)) break;
-        const uint32_t drop = ((state ? g.drop_if_bad : g.drop_if_good) >> b) & 1u;
-        word |= (drop ^ 1u) << b;
-        state = ((state ? g.stay_bad_if_bad : g.to_bad_if_good) >> b) & 1u;
+    const uint64_t n_words = row_words * W;
+    const uint64_t j0 = (uint64_t)blockIdx.x * kGeWordsPerBlock + (threadIdx.x >> 5) * kGeWordsPerWarp;
+    GeLane g[kGeWordsPerWarp];
+    uint32_t f = kFnIdentity;
+#pragma unroll
+    for (int q = 0; q < kGeWordsPerWarp; ++q) {
+        if (j0 + q < n_words) {
+            g[q] = ge_word(m, dk, j0 + q, C, row_words);
+            f = fn_after(g[q].word_fn, fn_after(g[q].reset, f));
+        }
     }
-    delivered[j] = word;
+    uint32_t total;
+    const uint32_t before = ge_block_prefix(f, &total);
+    uint32_t state = fn_apply(before, block_state[blockIdx.x]);       // state in which the warp's first word is entered
+#pragma unroll
+    for (int q = 0; q < kGeWordsPerWarp; ++q) {
+        if (j0 + q < n_words) {
+            state = fn_apply(g[q].reset, state);
+            const uint32_t mine = fn_apply(g[q].before, state);      // the packet is judged in the state it is sent in
+            const bool alive = g[q].valid && !(mine ? g[q].drop_if_bad : g[q].drop_if_good);
+            const uint32_t word = __ballot_sync(0xFFFFFFFFu, alive);
+            if ((threadIdx.x & 31) == 0) delivered[j0 + q] = word;
+            state = fn_apply(g[q].word_fn, state);
+        }
+    }
 }
 
 // ------------------------------------------------------------------------------------------------ arrival order
@@ -178,38 +210,56 @@ struct PermParams {
     uint32_t M;
 };
 
-__device__ __forceinline__ uint32_t permute(const PermParams& pp, const DrawKey& dk, uint32_t a)
+__device__ __forceinline__ uint32_t feistel(const PermParams& pp, const DrawKey& dk, uint32_t x)
 {
-    uint32_t x = a;
-    do {   // a cycle of the permutation of [0, 2^b) that starts below M returns below M: the walk ends
-        uint32_t L = x >> pp.half, R = x & pp.mask;
+    uint32_t L = x >> pp.half, R = x & pp.mask;
 #pragma unroll
-        for (uint32_t r = 0; r < 4; ++r) {
-            const uint32_t F = philox4x32_10(make_uint4(R, r, kStreamPerm | dk.attempt8, dk.round), dk.key).x & pp.mask;
-            const uint32_t nl = R;
-            R = L ^ F;
-            L = nl;
-        }
-        x = (L << pp.half) | R;
-    } while (x >= pp.M);
-    return x;
+    for (uint32_t r = 0; r < 4; ++r) {
+        const uint32_t F = philox4x32_10(make_uint4(R, r, kStreamPerm | dk.attempt8, dk.round), dk.key).x & pp.mask;
+        const uint32_t nl = R;
+        R = L ^ F;
+        L = nl;
+    }
+    return (L << pp.half) | R;
 }
 
-__global__ void __launch_bounds__(kPermThreads)
+__global__ void __launch_bounds__(kPermWalkers)
 k_perm_flags(PermParams pp, DrawKey dk, uint64_t C, uint64_t row_words, const uint32_t* __restrict__ delivered,
              uint32_t* __restrict__ perm_flag, uint32_t* __restrict__ block_count)
 {
-    const uint32_t a = blockIdx.x * kPermThreads + threadIdx.x;
-    int flag = 0;
-    if (a < pp.M) {
-        const uint32_t p = permute(pp, dk, a);
-        const uint32_t w = (uint32_t)(p / C);
-        const uint64_t seq = p - (uint64_t)w * C;
-        flag = (__ldg(&delivered[(uint64_t)w * row_words + (seq >> 5)]) >> (seq & 31)) & 1u;
-        perm_flag[a] = p | ((uint32_t)flag << 31);
+    constexpr uint32_t K = kPermThreads / kPermWalkers;
+    __shared__ uint32_t s_warp[kPermWalkers / 32];
+    const uint32_t a0 = blockIdx.x * kPermThreads + threadIdx.x * K;
+    const uint32_t n = a0 < pp.M ? min(K, pp.M - a0) : 0;
+    uint32_t out[K];
+#pragma unroll
+    for (uint32_t q = 0; q < K; ++q) out[q] = 0;
+    uint32_t k = 0, x = a0, flags = 0;
+    while (k < n) {       // every walk ends: a cycle of the permutation of [0, 2^b) that starts below M returns below M
+        x = feistel(pp, dk, x);
+        if (x < pp.M) {
+            const uint32_t w = (uint32_t)(x / C);
+            const uint64_t seq = x - (uint64_t)w * C;
+            const uint32_t flag = (__ldg(&delivered[(uint64_t)w * row_words + (seq >> 5)]) >> (seq & 31)) & 1u;
+#pragma unroll
+            for (uint32_t q = 0; q < K; ++q)
+                if (q == k) out[q] = x | (flag << 31);
+            flags += flag;
+            ++k;
+            x = a0 + k;
+        }
     }
-    const int n = __syncthreads_count(flag);
-    if (threadIdx.x == 0) block_count[blockIdx.x] = (uint32_t)n;
+#pragma unroll
+    for (uint32_t q = 0; q < K; ++q)
+        if (q < n) perm_flag[a0 + q] = out[q];
+    flags = __reduce_add_sync(0xFFFFFFFFu, flags);
+    if ((threadIdx.x & 31) == 0) s_warp[threadIdx.x >> 5] = flags;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t total = 0;
+        for (int q = 0; q < kPermWalkers / 32; ++q) total += s_warp[q];
+        block_count[blockIdx.x] = total;
+    }
 }
 
 // One block: exclusive prefix sum of the per-block survivor counts (in place) and the total.
@@ -269,7 +319,7 @@ static WorkspaceLayout layout(const dblp_plan* p)
     WorkspaceLayout l{};
     auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
     l.n_perm_blocks = (uint32_t)((p->M + kPermThreads - 1) / kPermThreads);
-    l.n_ge_blocks = (uint32_t)((p->row_words * p->W + kGeThreads - 1) / kGeThreads);
+    l.n_ge_blocks = (uint32_t)((p->row_words * p->W + kGeWordsPerBlock - 1) / kGeWordsPerBlock);
     l.perm_flag = 0;
     l.block_count = up(l.perm_flag + p->M * sizeof(uint32_t));
     l.ge_fn = up(l.block_count + (size_t)l.n_perm_blocks * sizeof(uint32_t));
@@ -337,7 +387,7 @@ extern "C" int dblp_apply_loss(const dblp_plan_t* plan, const dblp_loss_model_t*
     pp.half = bits / 2;
     pp.mask = (1u << pp.half) - 1u;
     pp.M = (uint32_t)plan->M;
-    k_perm_flags<<<l.n_perm_blocks, kPermThreads, 0, s>>>(pp, dk, plan->C, plan->row_words, delivered_bits, perm_flag, block_count);
+    k_perm_flags<<<l.n_perm_blocks, kPermWalkers, 0, s>>>(pp, dk, plan->C, plan->row_words, delivered_bits, perm_flag, block_count);
     DBLP_LAUNCHED();
     k_count_scan<<<1, kScanThreads, 0, s>>>(block_count, l.n_perm_blocks, n_arrived_dev);
     DBLP_LAUNCHED();
