@@ -55,7 +55,7 @@ typedef struct {
 } orc_loss_t;
 
 typedef struct {
-    uint64_t n_arrived, n_accepted, n_dup, n_stale, n_invalid;
+    uint64_t n_arrived, n_accepted, n_dup, n_stale, n_invalid, n_late;
     uint32_t status, pad;
 } orc_counters_t;
 
@@ -217,9 +217,15 @@ static void set_bit(uint32_t* bm, uint64_t C, uint32_t w, uint64_t seq)
  *                drop iff u0 < (Bad ? t_drop_bad : t_drop_good);
  *                then Bad stays Bad unless u1 < t_bg, Good turns Bad iff u1 < t_gb.
  * Output: delivered bitmap (1 = survived), rows per worker.
+ * A retransmission attempt sends only the chunks the latest bitmap reports
+ * missing (Algorithm 1: "for each unsent chunk"; Section III-B).  `sent` (same
+ * layout as the output, NULL = everything) is that set: a chunk that is not
+ * sent cannot arrive, and the burst chain, which models the channel while
+ * packets cross it, advances only over the packets that are sent.
  * ------------------------------------------------------------------------- */
-int dblp_oracle_loss_mask(const orc_loss_t* m, uint64_t C, uint32_t W, uint64_t seed, uint32_t round,
-                          uint32_t attempt, uint32_t* delivered, uint64_t* window_start_out)
+int dblp_oracle_loss_mask_sent(const orc_loss_t* m, uint64_t C, uint32_t W, uint64_t seed, uint32_t round,
+                               uint32_t attempt, const uint32_t* sent, uint32_t* delivered,
+                               uint64_t* window_start_out)
 {
     if (!m || !delivered || C == 0 || W == 0) return ORC_EINVAL;
     memset(delivered, 0, sizeof(uint32_t) * row_words(C) * W);
@@ -238,6 +244,7 @@ int dblp_oracle_loss_mask(const orc_loss_t* m, uint64_t C, uint32_t W, uint64_t 
             bad = (uint64_t)u[0] < m->t_init_bad;
         }
         for (uint64_t seq = 0; seq < C; ++seq) {
+            if (sent && !get_bit(sent, C, w, seq)) continue;
             uint64_t id = (uint64_t)w * C + seq;
             draw(seed, id, STREAM_PACKET, attempt, round, u);
             int drop;
@@ -258,6 +265,21 @@ int dblp_oracle_loss_mask(const orc_loss_t* m, uint64_t C, uint32_t W, uint64_t 
         }
     }
     return ORC_OK;
+}
+
+int dblp_oracle_loss_mask(const orc_loss_t* m, uint64_t C, uint32_t W, uint64_t seed, uint32_t round,
+                          uint32_t attempt, uint32_t* delivered, uint64_t* window_start_out)
+{
+    return dblp_oracle_loss_mask_sent(m, C, W, seed, round, attempt, NULL, delivered, window_start_out);
+}
+
+/* What the sender retransmits after a bitmap reply: every chunk whose bit is 0. */
+void dblp_oracle_missing_bits(uint64_t C, uint32_t W, const uint32_t* bitmap, uint32_t* sent)
+{
+    memset(sent, 0, sizeof(uint32_t) * row_words(C) * W);
+    for (uint32_t w = 0; w < W; ++w)
+        for (uint64_t seq = 0; seq < C; ++seq)
+            if (!get_bit(bitmap, C, w, seq)) set_bit(sent, C, w, seq);
 }
 
 /* ---------------------------------------------------------------------------
@@ -326,11 +348,18 @@ int dblp_oracle_arrival(uint64_t C, uint32_t W, uint64_t seed, uint32_t round, u
  * continue the same round (Section III-B: retransmission works from the most
  * recent bitmap).  The arrival number of entry a is counters->n_arrived (as it
  * stood before the call) + a.
+ * With early_stop (Algorithm 2, the branch without a probe: "if the
+ * loss-tolerance threshold is satisfied, send stop"), each worker's receiver
+ * stops the moment its own missing / total <= p holds (total = C, one bitmap
+ * per worker stream); whatever that worker delivers afterwards, valid and of
+ * this round, is late and ignored.  The integrity and round checks come first,
+ * as they do for a running receiver.
  * ------------------------------------------------------------------------- */
-int dblp_oracle_book(const uint64_t* numel, uint32_t T, uint32_t elem_size, uint32_t payload_bytes,
-                     uint32_t W, const orc_hdr_t* hdr_ring, uint64_t n_slots,
-                     const uint32_t* arrival, uint64_t n_arrived, uint32_t round,
-                     uint32_t* bitmap, uint32_t* slot_of, uint32_t* first_arrival, orc_counters_t* cnt)
+int dblp_oracle_book_stop(const uint64_t* numel, uint32_t T, uint32_t elem_size, uint32_t payload_bytes,
+                          uint32_t W, const orc_hdr_t* hdr_ring, uint64_t n_slots,
+                          const uint32_t* arrival, uint64_t n_arrived, uint32_t round,
+                          int early_stop, uint32_t bound_ppm,
+                          uint32_t* bitmap, uint32_t* slot_of, uint32_t* first_arrival, orc_counters_t* cnt)
 {
     uint64_t* base = (uint64_t*)malloc(sizeof(uint64_t) * T);
     uint64_t* cb = (uint64_t*)malloc(sizeof(uint64_t) * ((size_t)T + 1));
@@ -339,6 +368,10 @@ int dblp_oracle_book(const uint64_t* numel, uint32_t T, uint32_t elem_size, uint
     if (rc) { free(base); free(cb); return rc; }
     uint64_t E = payload_bytes / elem_size, C = cb[T];
     uint64_t first = cnt->n_arrived;
+    uint64_t* got = (uint64_t*)calloc(W, sizeof(uint64_t));          /* chunks received so far, per worker */
+    if (!got) { free(base); free(cb); return ORC_EINVAL; }
+    for (uint32_t w = 0; w < W; ++w)
+        for (uint64_t s = 0; s < C; ++s) got[w] += (uint64_t)get_bit(bitmap, C, w, s);
     for (uint64_t a = 0; a < n_arrived; ++a) {
         cnt->n_arrived++;
         uint64_t slot = arrival[a];
@@ -355,14 +388,25 @@ int dblp_oracle_book(const uint64_t* numel, uint32_t T, uint32_t elem_size, uint
         }
         if (!valid) { cnt->n_invalid++; continue; }
         if (h->round != round) { cnt->n_stale++; continue; }
+        if (early_stop && (C - got[h->worker]) * 1000000ull <= (uint64_t)bound_ppm * C) { cnt->n_late++; continue; }
         if (get_bit(bitmap, C, h->worker, h->seq)) { cnt->n_dup++; continue; }
         set_bit(bitmap, C, h->worker, h->seq);
         slot_of[(uint64_t)h->worker * C + h->seq] = (uint32_t)slot;
         first_arrival[(uint64_t)h->worker * C + h->seq] = (uint32_t)(first + a);
         cnt->n_accepted++;
+        got[h->worker]++;
     }
-    free(base); free(cb);
+    free(base); free(cb); free(got);
     return ORC_OK;
+}
+
+int dblp_oracle_book(const uint64_t* numel, uint32_t T, uint32_t elem_size, uint32_t payload_bytes,
+                     uint32_t W, const orc_hdr_t* hdr_ring, uint64_t n_slots,
+                     const uint32_t* arrival, uint64_t n_arrived, uint32_t round,
+                     uint32_t* bitmap, uint32_t* slot_of, uint32_t* first_arrival, orc_counters_t* cnt)
+{
+    return dblp_oracle_book_stop(numel, T, elem_size, payload_bytes, W, hdr_ring, n_slots, arrival, n_arrived, round,
+                                 0, 0, bitmap, slot_of, first_arrival, cnt);
 }
 
 /* bf16 -> fp32 is exact: the 16 bits are the top half of the fp32 pattern. */

@@ -26,10 +26,11 @@ class LossModel(C.Structure):
 
 class Counters(C.Structure):
     _fields_ = [("n_arrived", C.c_uint64), ("n_accepted", C.c_uint64), ("n_dup", C.c_uint64),
-                ("n_stale", C.c_uint64), ("n_invalid", C.c_uint64), ("status", C.c_uint32), ("pad", C.c_uint32)]
+                ("n_stale", C.c_uint64), ("n_invalid", C.c_uint64), ("n_late", C.c_uint64), ("status", C.c_uint32),
+                ("pad", C.c_uint32)]
 
     def as_dict(self):
-        return {k: int(getattr(self, k)) for k in ("n_arrived", "n_accepted", "n_dup", "n_stale", "n_invalid")}
+        return {k: int(getattr(self, k)) for k in ("n_arrived", "n_accepted", "n_dup", "n_stale", "n_invalid", "n_late")}
 
 
 _lib = None
@@ -129,12 +130,22 @@ class Plan:
                                            _p(h), C.byref(b)), "header_at")
         return h[0], int(b.value)
 
-    def loss_mask(self, model, seed, rnd, attempt=0):
+    def loss_mask(self, model, seed, rnd, attempt=0, sent=None):
+        """sent: bitmap of the chunks that are transmitted in this attempt (None = all)."""
         d = np.zeros(self.W * self.row_words, np.uint32)
         s0 = C.c_uint64()
-        _check(lib().dblp_oracle_loss_mask(C.byref(model), C.c_uint64(self.C), C.c_uint32(self.W), C.c_uint64(seed),
-                                           C.c_uint32(rnd), C.c_uint32(attempt), _p(d), C.byref(s0)), "loss_mask")
+        sp = None if sent is None else _p(np.ascontiguousarray(sent, np.uint32))
+        _check(lib().dblp_oracle_loss_mask_sent(C.byref(model), C.c_uint64(self.C), C.c_uint32(self.W), C.c_uint64(seed),
+                                                C.c_uint32(rnd), C.c_uint32(attempt), sp, _p(d), C.byref(s0)),
+               "loss_mask")
         return d.reshape(self.W, self.row_words), int(s0.value)
+
+    def missing_bits(self, bitmap):
+        """The set a sender retransmits after a bitmap reply: chunks whose bit is 0."""
+        out = np.zeros((self.W, self.row_words), np.uint32)
+        lib().dblp_oracle_missing_bits(C.c_uint64(self.C), C.c_uint32(self.W),
+                                       _p(np.ascontiguousarray(bitmap, np.uint32)), _p(out))
+        return out
 
     def perm(self, seed, rnd, attempt, a, M=None):
         return int(lib().dblp_oracle_perm(self.M if M is None else M, seed, rnd, attempt, a))
@@ -154,14 +165,39 @@ class Plan:
                 "first_arrival": np.full(self.W * self.C, NONE, np.uint32),
                 "counters": Counters()}
 
-    def book(self, hdr, arrival, n_arrived, rnd, state):
+    def book(self, hdr, arrival, n_arrived, rnd, state, stop_ppm=None):
+        """stop_ppm: None = every arrival is examined; a tolerance in ppm = each worker's receiver stops as soon as
+        its own missing / total <= p holds (Algorithm 2) and later arrivals of that worker count as late."""
         hdr = np.ascontiguousarray(hdr)
         arrival = np.ascontiguousarray(arrival, np.uint32)
-        _check(lib().dblp_oracle_book(*self._args(), C.c_uint32(self.W), _p(hdr), C.c_uint64(len(hdr)),
-                                      _p(arrival), C.c_uint64(n_arrived), C.c_uint32(rnd), _p(state["bitmap"]),
-                                      _p(state["slot_of"]), _p(state["first_arrival"]),
-                                      C.byref(state["counters"])), "book")
+        _check(lib().dblp_oracle_book_stop(*self._args(), C.c_uint32(self.W), _p(hdr), C.c_uint64(len(hdr)),
+                                           _p(arrival), C.c_uint64(n_arrived), C.c_uint32(rnd),
+                                           C.c_int(0 if stop_ppm is None else 1),
+                                           C.c_uint32(0 if stop_ppm is None else stop_ppm), _p(state["bitmap"]),
+                                           _p(state["slot_of"]), _p(state["first_arrival"]),
+                                           C.byref(state["counters"])), "book")
         return state
+
+    def round_until_stop(self, hdr, model, seed, rnd, bound_ppm, max_attempts, early_stop, state=None):
+        """Algorithm 1 + 2 as one loop: attempt k sends what the bitmap reports missing, the loss process and the
+        arrival order are redrawn with the attempt number, the receiver books the arrivals, and the round ends when
+        every worker's missing / total <= p (stop signal) or after max_attempts.  Returns (state, attempts used,
+        all_ok, per-attempt arrival counts)."""
+        state = self.new_state() if state is None else state
+        arrived = []
+        all_ok = 0
+        attempts = 0
+        for k in range(max_attempts):
+            sent = self.missing_bits(state["bitmap"])
+            d, _ = self.loss_mask(model, seed, rnd, k, sent)
+            arr, n = self.arrival(d, seed, rnd, k)
+            self.book(hdr, arr, n, rnd, state, bound_ppm if early_stop else None)
+            arrived.append(n)
+            attempts = k + 1
+            all_ok = self.check_bound(state["bitmap"], bound_ppm)[3]
+            if all_ok:
+                break
+        return state, attempts, all_ok, arrived
 
     def reduce(self, payload, state, mean=False):
         agg = np.empty(self.N, np.float32)

@@ -254,7 +254,7 @@ def test_book_counts_each_received_packet_exactly_once():
     p = orc.Plan([1000, 1, 352 * 40, 353, 7], 4, 1408, 4)
     hdr, pay, d, arr, n, st = _round(p, rand_grads(p, 4), orc.loss_model("iid", t_drop=wl.threshold(0.1)), 21)
     c = st["counters"].as_dict()
-    assert c == {"n_arrived": n, "n_accepted": n, "n_dup": 0, "n_stale": 0, "n_invalid": 0}
+    assert c == {"n_arrived": n, "n_accepted": n, "n_dup": 0, "n_stale": 0, "n_invalid": 0, "n_late": 0}
     assert np.array_equal(st["bitmap"], d)                      # received bitmap = delivered mask
     assert popcount(st["bitmap"]) == n                          # loss fraction = popcount of the mask
     sel = st["slot_of"] != orc.NONE
@@ -283,7 +283,7 @@ def test_book_drops_stale_duplicate_and_invalid_packets():
     arrival = np.array([5, 0, M + 0, M + 1, M + 2, M + 3, M + 4, M + 5, M + 6, M + 7, M + 8, 1, 5, M + 2],
                        np.uint32)                               # M+8 is outside the ring
     st = p.book(ring, arrival, len(arrival), 3, p.new_state())
-    assert st["counters"].as_dict() == {"n_arrived": 14, "n_accepted": 3, "n_dup": 3, "n_stale": 2, "n_invalid": 6}
+    assert st["counters"].as_dict() == {"n_arrived": 14, "n_accepted": 3, "n_dup": 3, "n_stale": 2, "n_invalid": 6, "n_late": 0}
     assert popcount(st["bitmap"]) == 3
     assert st["slot_of"][5] == 5 and st["first_arrival"][5] == 0          # first arrival keeps the slot
     # a duplicate that arrives BEFORE the original wins the slot instead
@@ -292,7 +292,7 @@ def test_book_drops_stale_duplicate_and_invalid_packets():
     # continuing the round: arrival numbers go on counting, earlier attempt keeps its slots
     st = p.book(ring, np.array([5, 7], np.uint32), 2, 3, st)
     assert st["slot_of"][5] == M + 2 and st["slot_of"][7] == 7 and st["first_arrival"][7] == 3
-    assert st["counters"].as_dict() == {"n_arrived": 4, "n_accepted": 2, "n_dup": 2, "n_stale": 0, "n_invalid": 0}
+    assert st["counters"].as_dict() == {"n_arrived": 4, "n_accepted": 2, "n_dup": 2, "n_stale": 0, "n_invalid": 0, "n_late": 0}
 
 
 # ------------------------------------------------------------------------------------------------ reduce
