@@ -203,7 +203,7 @@ def run_gpu(args):
         grads_host = [g.cpu().pin_memory() for g in grads]
         grads_dev = torch.empty(work.W * work.N, dtype=plan.torch_dtype, device=dev)
         agg_host = torch.empty(work.N, dtype=torch.float32).pin_memory()
-        cnt_host = torch.zeros(6, dtype=torch.int64).pin_memory()
+        cnt_host = torch.zeros(7, dtype=torch.int64).pin_memory()
         small = [torch.zeros(work.W, dtype=torch.int32).pin_memory() for _ in range(2)]
         ok_host = torch.zeros(work.W, dtype=torch.uint8).pin_memory()
         all_host = torch.zeros(1, dtype=torch.int32).pin_memory()
@@ -231,7 +231,7 @@ def run_gpu(args):
             ms_e2e = float(t.item())
         e2e = {"value": world * bytes_["total"] / ms_e2e / 1e6, "unit": "GB/s", "ms_per_step": ms_e2e, "steps": Ke,
                "h2d_bytes_per_step": work.W * work.N * work.elem_size,
-               "d2h_bytes_per_step": work.N * 4 + 48 + work.W * 9 + 4}
+               "d2h_bytes_per_step": work.N * 4 + 56 + work.W * 9 + 4}
         del grads_host, grads_dev
 
     cpu = None

@@ -85,6 +85,7 @@ typedef struct {
     uint64_t n_dup;      /* valid packets of this round whose chunk had already arrived */
     uint64_t n_stale;    /* valid packets of another round (Section III-A: dropped) */
     uint64_t n_invalid;  /* slot outside the ring, or header contradicting the plan (Algorithm 2 integrity check) */
+    uint64_t n_late;     /* valid packets of this round that came after their worker's receiver had stopped */
     uint32_t status;     /* bit 0: arrival numbers exceeded 32 bits */
     uint32_t pad;
 } dblp_counters_t;
@@ -135,6 +136,19 @@ int dblp_apply_loss(const dblp_plan_t* plan, const dblp_loss_model_t* model, uin
                     uint32_t attempt, uint32_t* delivered_bits, uint32_t* arrival, uint64_t* n_arrived_dev, void* ws,
                     size_t ws_bytes, void* stream);
 
+/* ---- retransmission attempts (Algorithm 1: "for each unsent chunk ... send"; Section III-B: the sender retransmits
+ * from the most recent bitmap) -------------------------------------------------------------------------------------
+ * dblp_missing_bits: sent_bits <- the chunks whose bit is 0 in recv_bitmap (padding bits stay 0): what a sender
+ * transmits after a bitmap reply.  Same layout as the bitmaps.
+ * dblp_apply_loss_resend: dblp_apply_loss restricted to the chunks in sent_bits (NULL = all, which is
+ * dblp_apply_loss): a chunk that is not sent cannot arrive, and the burst chain, which models the channel while
+ * packets cross it, advances only over the packets that are sent.  Draws are keyed by (packet id, attempt), so the
+ * fate of a sent packet under a memoryless process does not depend on what else is sent. */
+int dblp_missing_bits(const dblp_plan_t* plan, const uint32_t* recv_bitmap, uint32_t* sent_bits, void* stream);
+int dblp_apply_loss_resend(const dblp_plan_t* plan, const dblp_loss_model_t* model, uint64_t seed, uint32_t round,
+                           uint32_t attempt, const uint32_t* sent_bits, uint32_t* delivered_bits, uint32_t* arrival,
+                           uint64_t* n_arrived_dev, void* ws, size_t ws_bytes, void* stream);
+
 /* ---- apply_loss without any allocation (the paper has no counterpart: this entry point exists for the sake of
  * callers, not of the protocol) ---------------------------------------------------------------------------------
  * Same results as dblp_apply_loss, bit for bit, but the scratch is a fixed array inside the library's own device
@@ -180,6 +194,19 @@ int dblp_aggregate_book(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, uin
                         uint64_t* slot_key, dblp_counters_t* counters, void* stream);
 int dblp_aggregate_reduce(const dblp_plan_t* plan, const void* payload_ring, const uint64_t* slot_key, float* agg_out,
                           uint32_t flags, void* stream);
+
+/* ---- bookkeeping with early stop (Algorithm 2, the branch without a probe: "if the loss-tolerance threshold is
+ * satisfied, send stop") ------------------------------------------------------------------------------------------
+ * As dblp_aggregate_book, but each worker's receiver stops the moment its own missing / C <= bound_ppm / 10^6 holds
+ * (one bitmap per worker stream): of a worker's valid packets of this round, taken in arrival order, only those up
+ * to and including the one that satisfies the threshold are booked; the rest count as n_late and leave no trace.
+ * Integrity and round checks come first, as for a running receiver.  The result equals a sequential walk over the
+ * arrival list.  Needs W <= 4096 and a workspace of dblp_stop_workspace_bytes(arrival_cap) bytes, 256-byte aligned. */
+int dblp_stop_workspace_bytes(const dblp_plan_t* plan, uint64_t arrival_cap, size_t* bytes);
+int dblp_aggregate_book_stop(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, uint64_t n_slots,
+                             const uint32_t* arrival, const uint64_t* n_arrived_dev, uint64_t arrival_cap,
+                             uint32_t round, uint32_t bound_ppm, uint32_t* recv_bitmap, uint64_t* slot_key,
+                             dblp_counters_t* counters, void* ws, size_t ws_bytes, void* stream);
 int dblp_aggregate(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, const void* payload_ring, uint64_t n_slots,
                    const uint32_t* arrival, const uint64_t* n_arrived_dev, uint64_t arrival_cap, uint32_t round,
                    uint32_t* recv_bitmap, uint64_t* slot_key, dblp_counters_t* counters, float* agg_out,
@@ -230,8 +257,9 @@ typedef struct {
     uint32_t* missing_cnt;     /* W * B */
     uint8_t* ok;               /* W * B */
     uint32_t* all_ok;          /* 1 */
-    void* ws;
+    void* ws;                  /* max(dblp_workspace_bytes, dblp_stop_workspace_bytes(M)) when dblp_round_until_stop uses it */
     size_t ws_bytes;
+    uint32_t* sent_bits;       /* W * row_words; used by dblp_round_until_stop only */
 } dblp_device_buffers_t;
 
 int dblp_round_host(const dblp_plan_t* plan, const void* const* grads_host, const dblp_loss_model_t* model,
@@ -239,6 +267,18 @@ int dblp_round_host(const dblp_plan_t* plan, const void* const* grads_host, cons
                     const dblp_device_buffers_t* dev, float* agg_host, dblp_counters_t* counters_host,
                     uint32_t* recv_cnt_host, uint32_t* missing_cnt_host, uint8_t* ok_host, uint32_t* all_ok_host,
                     void* stream);
+
+/* ---- one round's control loop (Algorithms 1 + 2 together; HOST-blocking) ----------------------------------------------
+ * After dblp_round_reset and dblp_packetize: attempt k = 0, 1, ... transmits what the bitmap reports missing
+ * (dblp_missing_bits), redraws loss and arrival order with the attempt number (dblp_apply_loss_resend), books the
+ * arrivals (dblp_aggregate_book, or dblp_aggregate_book_stop when early_stop != 0) and tests the tolerance
+ * (dblp_check_bound, one value for all).  The decision is read back after every attempt -- the protocol's
+ * probe / bitmap / stop exchange is a round trip -- and the loop ends when every worker passes or after max_attempts.
+ * Packets are read from ring slots 0 .. M-1.  *attempts_used and *all_ok_host are HOST outputs.  The masked reduce is
+ * left to the caller (dblp_aggregate_reduce). */
+int dblp_round_until_stop(const dblp_plan_t* plan, const dblp_loss_model_t* model, uint64_t seed, uint32_t round,
+                          uint32_t bound_ppm, uint32_t max_attempts, int early_stop, const dblp_device_buffers_t* dev,
+                          uint32_t* attempts_used, uint32_t* all_ok_host, void* stream);
 
 /* ---- diagnostics -----------------------------------------------------------------------------------------------*/
 const char* dblp_strerror(int status);

@@ -16,7 +16,7 @@ DBLP_LOSS_NONE, DBLP_LOSS_IID, DBLP_LOSS_GE, DBLP_LOSS_MICROBURST = 0, 1, 2, 3
 DBLP_SUM, DBLP_MEAN = 0, 1
 LOSS_KINDS = {"none": DBLP_LOSS_NONE, "iid": DBLP_LOSS_IID, "ge": DBLP_LOSS_GE, "microburst": DBLP_LOSS_MICROBURST}
 HDR_BYTES = 32
-COUNTER_FIELDS = ("n_arrived", "n_accepted", "n_dup", "n_stale", "n_invalid")
+COUNTER_FIELDS = ("n_arrived", "n_accepted", "n_dup", "n_stale", "n_invalid", "n_late")
 
 
 class dblp_loss_model_t(C.Structure):
@@ -28,13 +28,15 @@ class dblp_loss_model_t(C.Structure):
 
 class dblp_counters_t(C.Structure):
     _fields_ = [("n_arrived", C.c_uint64), ("n_accepted", C.c_uint64), ("n_dup", C.c_uint64),
-                ("n_stale", C.c_uint64), ("n_invalid", C.c_uint64), ("status", C.c_uint32), ("pad", C.c_uint32)]
+                ("n_stale", C.c_uint64), ("n_invalid", C.c_uint64), ("n_late", C.c_uint64), ("status", C.c_uint32),
+                ("pad", C.c_uint32)]
 
 
 class dblp_device_buffers_t(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("grads", "hdr_ring", "payload_ring", "delivered_bits", "arrival",
                                           "n_arrived", "recv_bitmap", "slot_key", "counters", "agg", "recv_cnt",
-                                          "missing_cnt", "ok", "all_ok", "ws")] + [("ws_bytes", C.c_size_t)]
+                                          "missing_cnt", "ok", "all_ok", "ws")] + [("ws_bytes", C.c_size_t),
+                                                                                   ("sent_bits", C.c_void_p)]
 
 
 class DblpError(RuntimeError):
@@ -47,6 +49,8 @@ class DblpError(RuntimeError):
 _lib = None
 EXPORTS = ("dblp_plan_create", "dblp_plan_destroy", "dblp_plan_query", "dblp_plan_tune_reduce", "dblp_workspace_bytes",
            "dblp_loss_model_from_rates", "dblp_packetize", "dblp_apply_loss", "dblp_apply_loss_static",
+           "dblp_apply_loss_resend", "dblp_missing_bits", "dblp_stop_workspace_bytes", "dblp_aggregate_book_stop",
+           "dblp_round_until_stop",
            "dblp_aggregate_book",
            "dblp_aggregate_reduce", "dblp_aggregate", "dblp_round_reset", "dblp_check_bound", "dblp_bound_ok", "dblp_clr",
            "dblp_select_bound", "dblp_round_host", "dblp_strerror", "dblp_last_error", "dblp_launch_count")
@@ -150,16 +154,20 @@ class Plan:
         """Device buffers of one round, sized from the plan (torch is the allocator)."""
         n_slots = self.M if n_slots is None else n_slots
         cap = self.M if arrival_cap is None else arrival_cap
+        stop_ws = C.c_size_t()
+        _check(lib().dblp_stop_workspace_bytes(self.handle, C.c_uint64(cap), C.byref(stop_ws)), "dblp_stop_workspace_bytes")
+        ws_bytes = max(self.workspace_bytes, int(stop_ws.value))
         u8, u32, i64 = torch.uint8, torch.int32, torch.int64
         z = lambda n, dt: torch.zeros(n, dtype=dt, device=device)
         return {
             "hdr_ring": z(n_slots * HDR_BYTES, u8), "payload_ring": torch.empty(n_slots * self.P, dtype=u8, device=device),
             "delivered_bits": z(self.W * self.row_words, u32), "arrival": z(cap, u32), "n_arrived": z(1, i64),
             "recv_bitmap": z(self.W * self.row_words, u32), "slot_key": z(self.W * self.C, i64),
-            "counters": z(6, i64), "agg": torch.empty(self.N, dtype=torch.float32, device=device),
+            "counters": z(7, i64), "agg": torch.empty(self.N, dtype=torch.float32, device=device),
             "recv_cnt": z(self.W * self.B, u32), "missing_cnt": z(self.W * self.B, u32),
             "ok": z(self.W * self.B, u8), "all_ok": z(1, u32),
-            "ws": z((self.workspace_bytes + 7) // 8, i64), "n_slots": n_slots, "arrival_cap": cap,
+            "ws": z((ws_bytes + 7) // 8, i64), "sent_bits": z(self.W * self.row_words, u32),
+            "n_slots": n_slots, "arrival_cap": cap,
         }
 
 
@@ -185,6 +193,48 @@ def dblp_apply_loss_static(plan, model, seed, round, attempt, delivered_bits, ar
     _check(lib().dblp_apply_loss_static(plan.handle, C.byref(model), C.c_uint64(seed), C.c_uint32(round),
                                         C.c_uint32(attempt), _ptr(delivered_bits), _ptr(arrival), _ptr(n_arrived_dev),
                                         _stream(stream)), "dblp_apply_loss_static")
+
+
+def dblp_missing_bits(plan, recv_bitmap, sent_bits, stream=None):
+    _check(lib().dblp_missing_bits(plan.handle, _ptr(recv_bitmap), _ptr(sent_bits), _stream(stream)), "dblp_missing_bits")
+
+
+def dblp_apply_loss_resend(plan, model, seed, round, attempt, sent_bits, delivered_bits, arrival, n_arrived_dev, ws,
+                           stream=None):
+    _check(lib().dblp_apply_loss_resend(plan.handle, C.byref(model), C.c_uint64(seed), C.c_uint32(round),
+                                        C.c_uint32(attempt), _ptr(sent_bits), _ptr(delivered_bits), _ptr(arrival),
+                                        _ptr(n_arrived_dev), _ptr(ws), C.c_size_t(ws.numel() * ws.element_size()),
+                                        _stream(stream)), "dblp_apply_loss_resend")
+
+
+def dblp_aggregate_book_stop(plan, hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, bound_ppm,
+                             recv_bitmap, slot_key, counters, ws, stream=None):
+    _check(lib().dblp_aggregate_book_stop(plan.handle, _ptr(hdr_ring), C.c_uint64(n_slots), _ptr(arrival),
+                                          _ptr(n_arrived_dev), C.c_uint64(arrival_cap), C.c_uint32(round),
+                                          C.c_uint32(bound_ppm), _ptr(recv_bitmap), _ptr(slot_key), _ptr(counters),
+                                          _ptr(ws), C.c_size_t(ws.numel() * ws.element_size()), _stream(stream)),
+           "dblp_aggregate_book_stop")
+
+
+def _device_buffers(dev, grads_dev=None):
+    b = dblp_device_buffers_t()
+    b.grads = grads_dev.data_ptr() if grads_dev is not None else 0
+    for name in ("hdr_ring", "payload_ring", "delivered_bits", "arrival", "n_arrived", "recv_bitmap", "slot_key",
+                 "counters", "agg", "recv_cnt", "missing_cnt", "ok", "all_ok", "ws", "sent_bits"):
+        setattr(b, name, dev[name].data_ptr())
+    b.ws_bytes = dev["ws"].numel() * dev["ws"].element_size()
+    return b
+
+
+def dblp_round_until_stop(plan, model, seed, round, bound_ppm, max_attempts, early_stop, dev, stream=None):
+    """Returns (attempts used, all_ok).  Blocks: the decision is read back after every attempt."""
+    b = _device_buffers(dev)
+    attempts, ok = C.c_uint32(), C.c_uint32()
+    _check(lib().dblp_round_until_stop(plan.handle, C.byref(model), C.c_uint64(seed), C.c_uint32(round),
+                                       C.c_uint32(bound_ppm), C.c_uint32(max_attempts), C.c_int(int(early_stop)),
+                                       C.byref(b), C.byref(attempts), C.byref(ok), _stream(stream)),
+           "dblp_round_until_stop")
+    return int(attempts.value), int(ok.value)
 
 
 def dblp_aggregate_book(plan, hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, recv_bitmap, slot_key,
@@ -238,12 +288,7 @@ def dblp_round_host(plan, grads_host, model, seed, round, bound_ppm, flags, dev,
     """grads_host: W host tensors (pinned recommended); dev: buffers from Plan.alloc_round; grads_dev: one device
     tensor of W*N elements; *_host: host tensors that receive the results (None to skip)."""
     ptrs = (C.c_void_p * plan.W)(*[g.data_ptr() for g in grads_host])
-    b = dblp_device_buffers_t()
-    b.grads = grads_dev.data_ptr()
-    for name in ("hdr_ring", "payload_ring", "delivered_bits", "arrival", "n_arrived", "recv_bitmap", "slot_key",
-                 "counters", "agg", "recv_cnt", "missing_cnt", "ok", "all_ok", "ws"):
-        setattr(b, name, dev[name].data_ptr())
-    b.ws_bytes = dev["ws"].numel() * dev["ws"].element_size()
+    b = _device_buffers(dev, grads_dev)
     _check(lib().dblp_round_host(plan.handle, ptrs, C.byref(model), C.c_uint64(seed), C.c_uint32(round),
                                  C.c_uint32(bound_ppm), C.c_uint32(flags), C.byref(b), _ptr(agg_host),
                                  _ptr(counters_host), _ptr(recv_cnt_host), _ptr(missing_cnt_host), _ptr(ok_host),
@@ -256,6 +301,6 @@ def dblp_launch_count():
 
 def counters_dict(counters_tensor):
     v = counters_tensor.cpu().tolist()
-    d = dict(zip(COUNTER_FIELDS, v[:5]))
-    d["status"] = v[5] & 0xFFFFFFFF
+    d = dict(zip(COUNTER_FIELDS, v[:6]))
+    d["status"] = v[6] & 0xFFFFFFFF
     return d

@@ -88,6 +88,233 @@ k_bitmap(const unsigned long long* __restrict__ slot_key, uint32_t* __restrict__
     if ((threadIdx.x & 31) == 0) recv_bitmap[(uint64_t)w * row_words + (c >> 5)] = word;
 }
 
+// ------------------------------------------------------------------------------------------------ early stop
+// Sequential meaning (Algorithm 2): walk the arrival list; a worker's receiver stops right after the packet that brings
+// its missing share down to the tolerance; what that worker delivers later is late.  In parallel: every valid packet of
+// this round first claims its cell exactly as in k_book (so "first of its cell" is settled by the atomic minimum);
+// then, per worker, the position of the need-th first-of-cell packet in arrival order is found with per-block counts
+// and one search block per worker; finally every entry compares its own position with its worker's stop position
+// and late first-of-cell entries give their cell back.
+constexpr int kStopChunk = 1024;        // arrival entries per counting block
+constexpr int64_t kNeverStops = (int64_t)1 << 62;
+
+__global__ void __launch_bounds__(256)
+k_row_counts(const uint32_t* __restrict__ bitmap, uint64_t row_words, uint32_t* __restrict__ got)
+{
+    __shared__ uint32_t s_warp[8];
+    const uint32_t* row = bitmap + (uint64_t)blockIdx.x * row_words;
+    uint32_t n = 0;
+    for (uint64_t k = threadIdx.x; k < row_words; k += 256) n += __popc(__ldg(&row[k]));
+    n = __reduce_add_sync(0xFFFFFFFFu, n);
+    if ((threadIdx.x & 31) == 0) s_warp[threadIdx.x >> 5] = n;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t t = 0;
+        for (int k = 0; k < 8; ++k) t += s_warp[k];
+        got[blockIdx.x] = t;
+    }
+}
+
+// Validation and claim as in k_book; records each entry's cell (kEmpty32 for invalid / stale entries) and counts only
+// what does not depend on the stop positions.
+__global__ void __launch_bounds__(kBookThreads)
+k_book_claim(const dblp_hdr_t* __restrict__ hdr_ring, uint64_t n_slots, const uint32_t* __restrict__ arrival,
+             const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap, uint32_t round,
+             unsigned long long* __restrict__ slot_key, dblp_counters_t* counters, uint32_t* __restrict__ cell_of,
+             const uint64_t* __restrict__ numel, const uint32_t* __restrict__ chunkbase,
+             uint32_t T, uint32_t W, uint64_t C, uint32_t E, uint32_t es)
+{
+    const uint64_t n = min(*n_arrived_dev, arrival_cap);
+    const uint64_t a = (uint64_t)blockIdx.x * kBookThreads + threadIdx.x;
+    if ((uint64_t)blockIdx.x * kBookThreads >= n) return;
+    const uint64_t first_number = counters->n_arrived;
+    int stale = 0, invalid = 0;
+    if (a < n) {
+        const uint32_t slot = __ldg(&arrival[a]);
+        bool valid = false;
+        uint4 h0 = make_uint4(0, 0, 0, 0), h1 = h0;
+        if (slot < n_slots) {
+            const uint4* hp = reinterpret_cast<const uint4*>(hdr_ring + slot);
+            h0 = __ldg(hp);
+            h1 = __ldg(hp + 1);
+            const uint64_t off = (uint64_t)h1.x | ((uint64_t)h1.y << 32);
+            if (h1.z < W && h0.w < T) {
+                const uint64_t nt = __ldg(&numel[h0.w]);
+                if (off < nt && off % E == 0) {
+                    const uint64_t len = min((uint64_t)E, nt - off);
+                    valid = (h0.z == len * es) && (h0.x == __ldg(&chunkbase[h0.w]) + off / E);
+                }
+            }
+        }
+        uint32_t cell = kEmpty32;
+        if (!valid) invalid = 1;
+        else if (h0.y != round) stale = 1;
+        else {
+            cell = (uint32_t)((uint64_t)h1.z * C + h0.x);
+            atomicMin(&slot_key[cell], ((first_number + a) << 32) | slot);
+        }
+        cell_of[a] = cell;
+    }
+    const int n_stale = __syncthreads_count(stale), n_inv = __syncthreads_count(invalid);
+    if (threadIdx.x == 0) {
+        if (n_stale) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_stale), (unsigned long long)n_stale);
+        if (n_inv) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_invalid), (unsigned long long)n_inv);
+    }
+}
+
+__device__ __forceinline__ bool is_first_of_cell(const unsigned long long* slot_key, uint32_t cell, uint64_t number)
+{
+    return (uint32_t)(slot_key[cell] >> 32) == (uint32_t)number;
+}
+
+// Per block of kStopChunk arrival entries: how many first-of-cell packets each worker has in it.
+__global__ void __launch_bounds__(256)
+k_stop_count(const uint32_t* __restrict__ cell_of, const unsigned long long* __restrict__ slot_key,
+             const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap, const dblp_counters_t* counters,
+             uint32_t W, uint64_t C, uint32_t* __restrict__ block_cnt)
+{
+    extern __shared__ uint32_t s_cnt[];      // W counters
+    for (uint32_t k = threadIdx.x; k < W; k += 256) s_cnt[k] = 0;
+    __syncthreads();
+    const uint64_t n = min(*n_arrived_dev, arrival_cap), first_number = counters->n_arrived;
+    const uint64_t a0 = (uint64_t)blockIdx.x * kStopChunk;
+    for (uint32_t k = threadIdx.x; k < kStopChunk; k += 256) {
+        const uint64_t a = a0 + k;
+        if (a >= n) break;
+        const uint32_t cell = cell_of[a];
+        if (cell != kEmpty32 && is_first_of_cell(slot_key, cell, first_number + a)) atomicAdd(&s_cnt[cell / C], 1u);
+    }
+    __syncthreads();
+    for (uint32_t k = threadIdx.x; k < W; k += 256) block_cnt[(uint64_t)blockIdx.x * W + k] = s_cnt[k];
+}
+
+// One block per worker: the arrival index at which that worker's receiver stops (-1: it had stopped before this call,
+// kNeverStops: it does not get there).
+__global__ void __launch_bounds__(256)
+k_stop_find(const uint32_t* __restrict__ cell_of, const unsigned long long* __restrict__ slot_key,
+            const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap, const dblp_counters_t* counters,
+            uint32_t W, uint64_t C, uint32_t bound_ppm, const uint32_t* __restrict__ got,
+            const uint32_t* __restrict__ block_cnt, uint32_t n_blocks, long long* __restrict__ stop_at)
+{
+    __shared__ uint32_t s_scan[256];
+    __shared__ uint32_t s_block, s_before;
+    const uint32_t w = blockIdx.x, tid = threadIdx.x;
+    const uint64_t need_total = C - ((uint64_t)bound_ppm * C) / 1000000ull;   // fewest chunks with missing/C <= p
+    const uint64_t have = got[w];
+    if (have >= need_total) {
+        if (tid == 0) stop_at[w] = -1;
+        return;
+    }
+    const uint32_t need = (uint32_t)(need_total - have);                        // this many more first-of-cell packets
+    const uint64_t n = min(*n_arrived_dev, arrival_cap), first_number = counters->n_arrived;
+
+    // which counting block holds the need-th one
+    const uint32_t per = (n_blocks + 255) / 256;
+    const uint32_t lo = min(n_blocks, tid * per), hi = min(n_blocks, lo + per);
+    uint32_t sum = 0;
+    for (uint32_t b = lo; b < hi; ++b) sum += block_cnt[(uint64_t)b * W + w];
+    s_scan[tid] = sum;
+    if (tid == 0) s_block = kEmpty32;
+    __syncthreads();
+    for (int d = 1; d < 256; d <<= 1) {
+        const uint32_t v = tid >= (uint32_t)d ? s_scan[tid - d] : 0;
+        __syncthreads();
+        s_scan[tid] += v;
+        __syncthreads();
+    }
+    uint32_t before = s_scan[tid] - sum;                                          // exclusive prefix of this thread
+    if (before < need && before + sum >= need) {                                  // exactly one thread, if any
+        for (uint32_t b = lo; b < hi; ++b) {
+            const uint32_t c = block_cnt[(uint64_t)b * W + w];
+            if (before + c >= need) { s_block = b; s_before = before; break; }
+            before += c;
+        }
+    }
+    __syncthreads();
+    if (s_block == kEmpty32) {
+        if (tid == 0) stop_at[w] = kNeverStops;
+        return;
+    }
+    // the exact entry inside that block: each thread owns four consecutive entries
+    const uint32_t rank = need - s_before;                                        // 1-based rank inside the block
+    const uint64_t a0 = (uint64_t)s_block * kStopChunk + tid * 4;
+    uint32_t flags = 0;
+    for (uint32_t k = 0; k < 4; ++k) {
+        const uint64_t a = a0 + k;
+        if (a < n) {
+            const uint32_t cell = cell_of[a];
+            if (cell != kEmpty32 && cell / C == w && is_first_of_cell(slot_key, cell, first_number + a)) flags |= 1u << k;
+        }
+    }
+    const uint32_t mine = __popc(flags);
+    __syncthreads();
+    s_scan[tid] = mine;
+    __syncthreads();
+    for (int d = 1; d < 256; d <<= 1) {
+        const uint32_t v = tid >= (uint32_t)d ? s_scan[tid - d] : 0;
+        __syncthreads();
+        s_scan[tid] += v;
+        __syncthreads();
+    }
+    const uint32_t excl = s_scan[tid] - mine;
+    if (excl < rank && excl + mine >= rank) {
+        uint32_t seen = excl;
+        for (uint32_t k = 0; k < 4; ++k) {
+            if ((flags >> k) & 1u) {
+                if (++seen == rank) { stop_at[w] = (long long)(a0 + k); break; }
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kBookThreads)
+k_stop_apply(const uint32_t* __restrict__ cell_of, unsigned long long* __restrict__ slot_key,
+             const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap, dblp_counters_t* counters, uint64_t C,
+             const long long* __restrict__ stop_at)
+{
+    const uint64_t n = min(*n_arrived_dev, arrival_cap);
+    const uint64_t a = (uint64_t)blockIdx.x * kBookThreads + threadIdx.x;
+    if ((uint64_t)blockIdx.x * kBookThreads >= n) return;
+    const uint64_t first_number = counters->n_arrived;
+    int accepted = 0, dup = 0, late = 0;
+    if (a < n) {
+        const uint32_t cell = cell_of[a];
+        if (cell != kEmpty32) {
+            const bool first = is_first_of_cell(slot_key, cell, first_number + a);
+            if ((long long)a > stop_at[cell / C]) {
+                late = 1;
+                if (first) slot_key[cell] = kEmpty64;       // only the claimant gives the cell back
+            } else if (first) accepted = 1;
+            else dup = 1;
+        }
+    }
+    const int n_acc = __syncthreads_count(accepted), n_dup = __syncthreads_count(dup), n_late = __syncthreads_count(late);
+    if (threadIdx.x == 0) {
+        if (n_acc) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_accepted), (unsigned long long)n_acc);
+        if (n_dup) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_dup), (unsigned long long)n_dup);
+        if (n_late) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_late), (unsigned long long)n_late);
+    }
+}
+
+struct StopLayout {
+    size_t cell_of, block_cnt, got, stop_at, total;
+    uint32_t n_blocks;
+};
+
+static StopLayout stop_layout(const dblp_plan* p, uint64_t arrival_cap)
+{
+    StopLayout l{};
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    l.n_blocks = (uint32_t)((arrival_cap + kStopChunk - 1) / kStopChunk);
+    l.cell_of = 0;
+    l.block_cnt = up(arrival_cap * sizeof(uint32_t));
+    l.got = up(l.block_cnt + (size_t)l.n_blocks * p->W * sizeof(uint32_t));
+    l.stop_at = up(l.got + (size_t)p->W * sizeof(uint32_t));
+    l.total = up(l.stop_at + (size_t)p->W * sizeof(long long));
+    return l;
+}
+
+
 // ------------------------------------------------------------------------------------------------ reduce
 __device__ __forceinline__ uint4 ld_payload16(const uint8_t* p)
 {
@@ -392,6 +619,59 @@ extern "C" int dblp_aggregate_book(const dblp_plan_t* plan, const dblp_hdr_t* hd
     const uint64_t cells = plan->row_words * 32 * plan->W;
     k_bitmap<<<(unsigned)((cells + 255) / 256), 256, 0, s>>>(reinterpret_cast<const unsigned long long*>(slot_key),
                                                            recv_bitmap, plan->W, plan->C, plan->row_words,
+                                                           n_arrived_dev, arrival_cap, counters);
+    DBLP_LAUNCHED();
+    return DBLP_OK;
+}
+
+extern "C" int dblp_stop_workspace_bytes(const dblp_plan_t* plan, uint64_t arrival_cap, size_t* bytes)
+{
+    DBLP_REQUIRE(plan && bytes, DBLP_EINVAL, "stop_workspace_bytes: null argument");
+    *bytes = stop_layout(plan, arrival_cap).total;
+    return DBLP_OK;
+}
+
+extern "C" int dblp_aggregate_book_stop(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, uint64_t n_slots,
+                                        const uint32_t* arrival, const uint64_t* n_arrived_dev, uint64_t arrival_cap,
+                                        uint32_t round, uint32_t bound_ppm, uint32_t* recv_bitmap, uint64_t* slot_key,
+                                        dblp_counters_t* counters, void* ws, size_t ws_bytes, void* stream)
+{
+    DBLP_REQUIRE(plan && hdr_ring && arrival && n_arrived_dev && recv_bitmap && slot_key && counters && ws, DBLP_EINVAL,
+                 "aggregate_book_stop: null argument");
+    DBLP_REQUIRE(aligned16(hdr_ring), DBLP_EALIGN, "aggregate_book_stop: header ring must be 16-byte aligned");
+    DBLP_REQUIRE((reinterpret_cast<uintptr_t>(ws) & 255u) == 0, DBLP_EALIGN, "aggregate_book_stop: workspace must be 256-byte aligned");
+    DBLP_REQUIRE(n_slots < 0xFFFFFFFFull && arrival_cap < (1ull << 32), DBLP_ECAPACITY, "aggregate_book_stop: ring or arrival list too long");
+    DBLP_REQUIRE(plan->W <= 4096, DBLP_ECAPACITY, "aggregate_book_stop: more than 4096 workers");
+    DBLP_REQUIRE(bound_ppm <= 1000000, DBLP_EINVAL, "aggregate_book_stop: tolerance above 100 %%");
+    const StopLayout l = stop_layout(plan, arrival_cap);
+    DBLP_REQUIRE(ws_bytes >= l.total, DBLP_ECAPACITY, "aggregate_book_stop: workspace of %zu bytes, %zu needed", ws_bytes, l.total);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint8_t* base = static_cast<uint8_t*>(ws);
+    uint32_t* cell_of = reinterpret_cast<uint32_t*>(base + l.cell_of);
+    uint32_t* block_cnt = reinterpret_cast<uint32_t*>(base + l.block_cnt);
+    uint32_t* got = reinterpret_cast<uint32_t*>(base + l.got);
+    long long* stop_at = reinterpret_cast<long long*>(base + l.stop_at);
+    unsigned long long* keys = reinterpret_cast<unsigned long long*>(slot_key);
+
+    k_row_counts<<<plan->W, 256, 0, s>>>(recv_bitmap, plan->row_words, got);
+    DBLP_LAUNCHED();
+    if (arrival_cap > 0) {
+        const unsigned grid = (unsigned)((arrival_cap + kBookThreads - 1) / kBookThreads);
+        k_book_claim<<<grid, kBookThreads, 0, s>>>(hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, keys, counters,
+                                                   cell_of, plan->d_numel, plan->d_chunkbase, plan->T, plan->W, plan->C,
+                                                   plan->E, plan->es);
+        DBLP_LAUNCHED();
+        k_stop_count<<<l.n_blocks, 256, plan->W * sizeof(uint32_t), s>>>(cell_of, keys, n_arrived_dev, arrival_cap, counters,
+                                                                        plan->W, plan->C, block_cnt);
+        DBLP_LAUNCHED();
+        k_stop_find<<<plan->W, 256, 0, s>>>(cell_of, keys, n_arrived_dev, arrival_cap, counters, plan->W, plan->C, bound_ppm,
+                                            got, block_cnt, l.n_blocks, stop_at);
+        DBLP_LAUNCHED();
+        k_stop_apply<<<grid, kBookThreads, 0, s>>>(cell_of, keys, n_arrived_dev, arrival_cap, counters, plan->C, stop_at);
+        DBLP_LAUNCHED();
+    }
+    const uint64_t cells = plan->row_words * 32 * plan->W;
+    k_bitmap<<<(unsigned)((cells + 255) / 256), 256, 0, s>>>(keys, recv_bitmap, plan->W, plan->C, plan->row_words,
                                                            n_arrived_dev, arrival_cap, counters);
     DBLP_LAUNCHED();
     return DBLP_OK;

@@ -32,7 +32,8 @@ struct LossParams {
 
 // ------------------------------------------------------------------------------------------------ memoryless kinds
 __global__ void __launch_bounds__(kLossThreads)
-k_loss_pointwise(LossParams m, DrawKey dk, uint32_t W, uint64_t C, uint64_t row_words, uint32_t* __restrict__ delivered)
+k_loss_pointwise(LossParams m, DrawKey dk, uint32_t W, uint64_t C, uint64_t row_words,
+                 const uint32_t* __restrict__ sent, uint32_t* __restrict__ delivered)
 {
     __shared__ uint64_t s_window_start;
     if (m.kind == DBLP_LOSS_MICROBURST) {
@@ -45,7 +46,7 @@ k_loss_pointwise(LossParams m, DrawKey dk, uint32_t W, uint64_t C, uint64_t row_
     const uint32_t w = (uint32_t)(i / row_bits);
     const uint64_t seq = i - (uint64_t)w * row_bits;
     bool alive = false;
-    if (seq < C) {
+    if (seq < C && (!sent || ((__ldg(&sent[(uint64_t)w * row_words + (seq >> 5)]) >> (seq & 31)) & 1u))) {
         uint64_t t = 0;
         if (m.kind == DBLP_LOSS_IID) t = m.t_drop;
         else if (m.kind == DBLP_LOSS_MICROBURST)
@@ -74,15 +75,16 @@ struct GeLane {
     bool valid, drop_if_good, drop_if_bad;
 };
 
-__device__ __forceinline__ GeLane ge_word(const LossParams& m, const DrawKey& dk, uint64_t j, uint64_t C, uint64_t row_words)
+__device__ __forceinline__ GeLane ge_word(const LossParams& m, const DrawKey& dk, const uint32_t* sent, uint64_t j, uint64_t C,
+                                          uint64_t row_words)
 {
     GeLane g;
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t w = (uint32_t)(j / row_words);
     const uint64_t k = j - (uint64_t)w * row_words;
     const uint64_t seq = k * 32 + lane;
-    g.valid = seq < C;
-    uint32_t fn = kFnIdentity;          // padding bits past the end of the row leave the state alone
+    g.valid = seq < C && (!sent || ((__ldg(&sent[j]) >> lane) & 1u));   // packets that are not sent leave the chain alone
+    uint32_t fn = kFnIdentity;          // so do the padding bits past the end of the row
     g.drop_if_good = g.drop_if_bad = false;
     if (g.valid) {
         const uint4 u = draw(dk, (uint64_t)w * C + seq, kStreamPacket);
@@ -126,14 +128,15 @@ __device__ __forceinline__ uint32_t ge_block_prefix(uint32_t warp_fn, uint32_t* 
 }
 
 __global__ void __launch_bounds__(kGeThreads)
-k_ge_partial(LossParams m, DrawKey dk, uint32_t W, uint64_t C, uint64_t row_words, uint8_t* __restrict__ block_fn)
+k_ge_partial(LossParams m, DrawKey dk, uint32_t W, uint64_t C, uint64_t row_words, const uint32_t* __restrict__ sent,
+             uint8_t* __restrict__ block_fn)
 {
     const uint64_t n_words = row_words * W;
     const uint64_t j0 = (uint64_t)blockIdx.x * kGeWordsPerBlock + (threadIdx.x >> 5) * kGeWordsPerWarp;
     uint32_t f = kFnIdentity;
     for (int q = 0; q < kGeWordsPerWarp; ++q) {
         if (j0 + q < n_words) {
-            const GeLane g = ge_word(m, dk, j0 + q, C, row_words);
+            const GeLane g = ge_word(m, dk, sent, j0 + q, C, row_words);
             f = fn_after(g.word_fn, fn_after(g.reset, f));
         }
     }
@@ -173,7 +176,7 @@ k_ge_block_states(const uint8_t* __restrict__ block_fn, uint8_t* __restrict__ bl
 }
 
 __global__ void __launch_bounds__(kGeThreads)
-k_ge_apply(LossParams m, DrawKey dk, uint32_t W, uint64_t C, uint64_t row_words,
+k_ge_apply(LossParams m, DrawKey dk, uint32_t W, uint64_t C, uint64_t row_words, const uint32_t* __restrict__ sent,
            const uint8_t* __restrict__ block_state, uint32_t* __restrict__ delivered)
 {
     const uint64_t n_words = row_words * W;
@@ -183,7 +186,7 @@ k_ge_apply(LossParams m, DrawKey dk, uint32_t W, uint64_t C, uint64_t row_words,
 #pragma unroll
     for (int q = 0; q < kGeWordsPerWarp; ++q) {
         if (j0 + q < n_words) {
-            g[q] = ge_word(m, dk, j0 + q, C, row_words);
+            g[q] = ge_word(m, dk, sent, j0 + q, C, row_words);
             f = fn_after(g[q].word_fn, fn_after(g[q].reset, f));
         }
     }
@@ -339,9 +342,10 @@ extern "C" int dblp_workspace_bytes(const dblp_plan_t* plan, size_t* bytes)
     return DBLP_OK;
 }
 
-extern "C" int dblp_apply_loss(const dblp_plan_t* plan, const dblp_loss_model_t* model, uint64_t seed, uint32_t round,
-                               uint32_t attempt, uint32_t* delivered_bits, uint32_t* arrival, uint64_t* n_arrived_dev,
-                               void* ws, size_t ws_bytes, void* stream)
+extern "C" int dblp_apply_loss_resend(const dblp_plan_t* plan, const dblp_loss_model_t* model, uint64_t seed,
+                                      uint32_t round, uint32_t attempt, const uint32_t* sent_bits,
+                                      uint32_t* delivered_bits, uint32_t* arrival, uint64_t* n_arrived_dev, void* ws,
+                                      size_t ws_bytes, void* stream)
 {
     DBLP_REQUIRE(plan && model && delivered_bits && arrival && n_arrived_dev && ws, DBLP_EINVAL, "apply_loss: null argument");
     DBLP_REQUIRE(model->kind <= DBLP_LOSS_MICROBURST, DBLP_EINVAL, "apply_loss: unknown loss kind %u", model->kind);
@@ -368,16 +372,17 @@ extern "C" int dblp_apply_loss(const dblp_plan_t* plan, const dblp_loss_model_t*
     DrawKey dk{make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)), attempt << 8, round};
 
     if (model->kind == DBLP_LOSS_GE) {
-        k_ge_partial<<<l.n_ge_blocks, kGeThreads, 0, s>>>(m, dk, plan->W, plan->C, plan->row_words, ge_fn);
+        k_ge_partial<<<l.n_ge_blocks, kGeThreads, 0, s>>>(m, dk, plan->W, plan->C, plan->row_words, sent_bits, ge_fn);
         DBLP_LAUNCHED();
         k_ge_block_states<<<1, kScanThreads, 0, s>>>(ge_fn, ge_state, l.n_ge_blocks);
         DBLP_LAUNCHED();
-        k_ge_apply<<<l.n_ge_blocks, kGeThreads, 0, s>>>(m, dk, plan->W, plan->C, plan->row_words, ge_state, delivered_bits);
+        k_ge_apply<<<l.n_ge_blocks, kGeThreads, 0, s>>>(m, dk, plan->W, plan->C, plan->row_words, sent_bits, ge_state,
+                                                       delivered_bits);
         DBLP_LAUNCHED();
     } else {
         const uint64_t threads = plan->row_words * 32 * plan->W;
         k_loss_pointwise<<<(unsigned)((threads + kLossThreads - 1) / kLossThreads), kLossThreads, 0, s>>>(
-            m, dk, plan->W, plan->C, plan->row_words, delivered_bits);
+            m, dk, plan->W, plan->C, plan->row_words, sent_bits, delivered_bits);
         DBLP_LAUNCHED();
     }
 
@@ -392,6 +397,37 @@ extern "C" int dblp_apply_loss(const dblp_plan_t* plan, const dblp_loss_model_t*
     k_count_scan<<<1, kScanThreads, 0, s>>>(block_count, l.n_perm_blocks, n_arrived_dev);
     DBLP_LAUNCHED();
     k_arrival_scatter<<<l.n_perm_blocks, kPermThreads, 0, s>>>(pp.M, perm_flag, block_count, arrival);
+    DBLP_LAUNCHED();
+    return DBLP_OK;
+}
+
+extern "C" int dblp_apply_loss(const dblp_plan_t* plan, const dblp_loss_model_t* model, uint64_t seed, uint32_t round,
+                               uint32_t attempt, uint32_t* delivered_bits, uint32_t* arrival, uint64_t* n_arrived_dev,
+                               void* ws, size_t ws_bytes, void* stream)
+{
+    return dblp_apply_loss_resend(plan, model, seed, round, attempt, nullptr, delivered_bits, arrival, n_arrived_dev, ws,
+                                  ws_bytes, stream);
+}
+
+namespace dblp {
+__global__ void __launch_bounds__(256)
+k_missing_bits(const uint32_t* __restrict__ bitmap, uint32_t* __restrict__ sent, uint64_t C, uint64_t row_words, uint64_t n_words)
+{
+    const uint64_t j = (uint64_t)blockIdx.x * 256 + threadIdx.x;
+    if (j >= n_words) return;
+    const uint64_t k = j % row_words;
+    uint32_t x = ~bitmap[j];
+    if (k == row_words - 1 && (C & 31)) x &= (1u << (C & 31)) - 1u;       // padding bits are not chunks
+    sent[j] = x;
+}
+}  // namespace dblp
+
+extern "C" int dblp_missing_bits(const dblp_plan_t* plan, const uint32_t* recv_bitmap, uint32_t* sent_bits, void* stream)
+{
+    DBLP_REQUIRE(plan && recv_bitmap && sent_bits, DBLP_EINVAL, "missing_bits: null argument");
+    const uint64_t n = plan->row_words * plan->W;
+    k_missing_bits<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(recv_bitmap, sent_bits, plan->C,
+                                                                                               plan->row_words, n);
     DBLP_LAUNCHED();
     return DBLP_OK;
 }

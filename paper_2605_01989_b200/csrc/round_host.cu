@@ -38,3 +38,38 @@ extern "C" int dblp_round_host(const dblp_plan_t* plan, const void* const* grads
     DBLP_CUDA(cudaStreamSynchronize(s));
     return DBLP_OK;
 }
+
+extern "C" int dblp_round_until_stop(const dblp_plan_t* plan, const dblp_loss_model_t* model, uint64_t seed, uint32_t round,
+                                     uint32_t bound_ppm, uint32_t max_attempts, int early_stop,
+                                     const dblp_device_buffers_t* dev, uint32_t* attempts_used, uint32_t* all_ok_host,
+                                     void* stream)
+{
+    DBLP_REQUIRE(plan && model && dev && attempts_used && all_ok_host, DBLP_EINVAL, "round_until_stop: null argument");
+    DBLP_REQUIRE(dev->sent_bits, DBLP_EINVAL, "round_until_stop: sent_bits buffer missing");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    *attempts_used = 0;
+    *all_ok_host = 0;
+    for (uint32_t k = 0; k < max_attempts; ++k) {
+        int rc = dblp_missing_bits(plan, dev->recv_bitmap, dev->sent_bits, s);
+        if (rc == DBLP_OK) rc = dblp_apply_loss_resend(plan, model, seed, round, k, dev->sent_bits, dev->delivered_bits,
+                                                      dev->arrival, dev->n_arrived, dev->ws, dev->ws_bytes, s);
+        if (rc == DBLP_OK) {
+            if (early_stop)
+                rc = dblp_aggregate_book_stop(plan, dev->hdr_ring, plan->M, dev->arrival, dev->n_arrived, plan->M, round,
+                                              bound_ppm, dev->recv_bitmap, dev->slot_key, dev->counters, dev->ws,
+                                              dev->ws_bytes, s);
+            else
+                rc = dblp_aggregate_book(plan, dev->hdr_ring, plan->M, dev->arrival, dev->n_arrived, plan->M, round,
+                                         dev->recv_bitmap, dev->slot_key, dev->counters, s);
+        }
+        if (rc == DBLP_OK) rc = dblp_check_bound(plan, dev->recv_bitmap, &bound_ppm, 1, dev->recv_cnt, dev->missing_cnt,
+                                                dev->ok, dev->all_ok, s);
+        if (rc != DBLP_OK) return rc;
+        // the stop / bitmap reply is a round trip of the protocol: the decision comes back to the host every attempt
+        DBLP_CUDA(cudaMemcpyAsync(all_ok_host, dev->all_ok, sizeof(uint32_t), cudaMemcpyDeviceToHost, s));
+        DBLP_CUDA(cudaStreamSynchronize(s));
+        *attempts_used = k + 1;
+        if (*all_ok_host) break;
+    }
+    return DBLP_OK;
+}

@@ -186,7 +186,7 @@ def test_round_host_entry_point_matches_the_oracle():
     g = H.GpuRound(w)
     grads_dev = torch.empty(w.W * w.N, dtype=torch.float32, device=H.DEV)
     agg_host = torch.empty(w.N, dtype=torch.float32).pin_memory()
-    cnt_host = torch.zeros(6, dtype=torch.int64).pin_memory()
+    cnt_host = torch.zeros(7, dtype=torch.int64).pin_memory()
     recv_host = torch.zeros(3, dtype=torch.int32).pin_memory()
     miss_host = torch.zeros(3, dtype=torch.int32).pin_memory()
     ok_host = torch.zeros(3, dtype=torch.uint8).pin_memory()
@@ -204,7 +204,7 @@ def test_round_host_entry_point_matches_the_oracle():
         assert recv_host.numpy().view(np.uint32).tolist() == o[0][:, 0].tolist()
         assert miss_host.numpy().view(np.uint32).tolist() == o[1][:, 0].tolist()
         assert ok_host.numpy().tolist() == o[2][:, 0].tolist() and int(all_host[0]) == o[3]
-        assert dict(zip(dblp.COUNTER_FIELDS, cnt_host.tolist()[:5])) == st["counters"].as_dict()
+        assert dict(zip(dblp.COUNTER_FIELDS, cnt_host.tolist()[:6])) == st["counters"].as_dict()
     g.close()
 
 
