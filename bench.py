@@ -234,6 +234,28 @@ def run_gpu(args):
                "d2h_bytes_per_step": work.N * 4 + 56 + work.W * 9 + 4}
         del grads_host, grads_dev
 
+    # the control loop under heavy i.i.d. bursts: attempts until every worker passes, low vs high tolerance
+    # (the mechanism behind the paper's latency tables; not part of the timed step)
+    round_loop = None
+    if rank == 0 and world == 1 and not args.no_round_loop:
+        p_low = bound
+        p_high = bound + 400000
+        round_loop = []
+        dblp.dblp_packetize(plan, grads, 7, buf["hdr_ring"], buf["payload_ring"])
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for burst in (0.6, 0.7, 0.8, 0.9):
+            m = dblp.loss_model("iid", t_drop=wl.threshold(burst))
+            row = {"loss": burst}
+            for name, ppm in (("p_low", p_low), ("p_high", p_high)):
+                dblp.dblp_round_reset(plan, buf["recv_bitmap"], buf["slot_key"], buf["counters"])
+                a.record()
+                attempts, ok = dblp.dblp_round_until_stop(plan, m, work.seed, 7, ppm, 400, True, buf)
+                b.record()
+                torch.cuda.synchronize()
+                row[name] = {"ppm": ppm, "attempts": attempts, "all_ok": ok, "ms": a.elapsed_time(b)}
+            row["attempt_ratio"] = row["p_low"]["attempts"] / max(1, row["p_high"]["attempts"])
+            round_loop.append(row)
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu = cpu_baseline(work, bytes_["total"])
@@ -261,7 +283,7 @@ def run_gpu(args):
         "roofline": {"kernel": "k_reduce", "bound": "hbm", "achieved": red_gbs, "peak": peak, "peak_kind": peak_kind,
                      "unit": "GB/s", "frac": red_gbs / peak, "traffic": TRAFFIC.get(work.name),
                      "algorithmic_bytes_per_launch": bytes_["reduce"], "ms_per_launch": stage_ms["reduce"]},
-        "clocks": clocks, "gpu_launches": launches, "e2e": e2e, "cpu_baseline": cpu,
+        "clocks": clocks, "gpu_launches": launches, "e2e": e2e, "cpu_baseline": cpu, "round_loop": round_loop,
     }
     print(json.dumps(out))
 
@@ -369,6 +391,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=30)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-round-loop", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = 5 if args.steps is None else args.steps
