@@ -195,6 +195,23 @@ int dblp_aggregate_book(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, uin
 int dblp_aggregate_reduce(const dblp_plan_t* plan, const void* payload_ring, const uint64_t* slot_key, float* agg_out,
                           uint32_t flags, void* stream);
 
+/* ---- masked reduce with fused extras ---------------------------------------------------------------------------------
+ * dblp_aggregate_reduce plus, in the same pass over the data:
+ *   norm (Eq. 1 needs the L2 norm of the aggregated gradient): norm_out[0] = sum of agg[i]^2 in fp64, norm_out[1] = its
+ *     square root.  Squares of fp32 values are exact in fp64; the additions follow a fixed tree (per thread, warp
+ *     shuffle, warps in order, tiles in a fixed order), so the result is reproducible for a given plan and within
+ *     about 64 ulp of the exactly rounded sum.  norm_scratch: dblp_norm_scratch_count() doubles (changes when
+ *     dblp_plan_tune_reduce changes the tile height).  Both NULL = off.
+ *   update (Algorithm 4, worker: w <- w - alpha * g): params[i] = params[i] - lr * agg[i], an fp32 multiply then an
+ *     fp32 subtract (no fused multiply-add), for every element; chunks nobody delivered leave params unchanged because
+ *     their aggregate is +0.  params: N fp32, in/out.  NULL = off.
+ * For the broadcast half of a round (Algorithm 3 "DBLP_SEND(mean)", Algorithm 4 "DBLP_RECV"), packetize the mean with a
+ * W = 1 plan, apply loss, book, and call this with params: the worker's reconstruction and its update in one pass. */
+int dblp_norm_scratch_count(const dblp_plan_t* plan, uint64_t* count);
+int dblp_aggregate_reduce_ex(const dblp_plan_t* plan, const void* payload_ring, const uint64_t* slot_key, float* agg_out,
+                             uint32_t flags, double* norm_scratch, double* norm_out, float* params, float lr,
+                             void* stream);
+
 /* ---- bookkeeping with early stop (Algorithm 2, the branch without a probe: "if the loss-tolerance threshold is
  * satisfied, send stop") ------------------------------------------------------------------------------------------
  * As dblp_aggregate_book, but each worker's receiver stops the moment its own missing / C <= bound_ppm / 10^6 holds

@@ -15,7 +15,7 @@ def build(force: bool = False) -> str:
     if not force and os.path.exists(OUT) and os.path.getmtime(OUT) >= os.path.getmtime(SRC):
         return OUT
     cmd = ["gcc", "-std=c99", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fopenmp", "-fPIC", "-shared",
-           "-Wall", "-Wextra", "-o", OUT, SRC]
+           "-Wall", "-Wextra", "-o", OUT, SRC, "-lm"]
     subprocess.run(cmd, check=True)
     return OUT
 

@@ -24,6 +24,7 @@
 #include <stddef.h>
 #include <string.h>
 #include <stdlib.h>
+#include <math.h>
 
 #define ORC_OK 0
 #define ORC_EINVAL (-1)
@@ -558,4 +559,39 @@ uint32_t dblp_oracle_select_bound(double norm_prev, double norm_curr, double eta
     uint32_t p = p_high_ppm;
     if (dblp_oracle_clr(norm_prev, norm_curr, eta)) p = p_low_ppm;
     return p;
+}
+
+/* ---------------------------------------------------------------------------
+ * L2 norm of the aggregated gradient (Eq. 1 compares ||G_prev|| with ||G_curr||;
+ * Section III-B: the L2 norm).  By definition ||G||^2 = sum_i g_i^2.  Each square
+ * of an fp32 value is exact in fp64; the sum is carried with Neumaier's
+ * compensated summation so that the result is the exactly rounded sum to within
+ * an ulp or two whatever N is -- the definition's value, not one particular
+ * order of additions.
+ * ------------------------------------------------------------------------- */
+int dblp_oracle_norm(const float* g, uint64_t n, double* sum_sq, double* norm)
+{
+    double s = 0.0, c = 0.0;
+    for (uint64_t i = 0; i < n; ++i) {
+        double x = (double)g[i] * (double)g[i];
+        double t = s + x;
+        if ((s >= 0 ? s : -s) >= x) c += (s - t) + x;
+        else c += (x - t) + s;
+        s = t;
+    }
+    *sum_sq = s + c;
+    *norm = sqrt(*sum_sq);      /* the C library's sqrt: correctly rounded by IEEE 754 */
+    return ORC_OK;
+}
+
+/* ---------------------------------------------------------------------------
+ * Worker update (Algorithm 4: w <- w - alpha * g_hat): one fp32 multiply, then
+ * one fp32 subtract, per element.
+ * ------------------------------------------------------------------------- */
+void dblp_oracle_sgd_apply(float* params, const float* g, float lr, uint64_t n)
+{
+    for (uint64_t i = 0; i < n; ++i) {
+        float step = lr * g[i];
+        params[i] = params[i] - step;
+    }
 }

@@ -241,3 +241,20 @@ def clr(norm_prev, norm_curr, eta=0.5):
 def select_bound(norm_prev, norm_curr, eta, p_low_ppm, p_high_ppm, at_epoch_start, first_iteration, current_ppm):
     return int(lib().dblp_oracle_select_bound(norm_prev, norm_curr, eta, p_low_ppm, p_high_ppm,
                                               int(at_epoch_start), int(first_iteration), current_ppm))
+
+
+def norm(g):
+    """(sum of squares, L2 norm) of a float32 array, fp64."""
+    g = np.ascontiguousarray(g, np.float32)
+    s, n = C.c_double(), C.c_double()
+    _check(lib().dblp_oracle_norm(_p(g), C.c_uint64(g.size), C.byref(s), C.byref(n)), "norm")
+    return float(s.value), float(n.value)
+
+
+def sgd_apply(params, g, lr):
+    """params - lr * g per element in fp32 (multiply, then subtract); returns a new array."""
+    out = np.ascontiguousarray(params, np.float32).copy()
+    g = np.ascontiguousarray(g, np.float32)
+    assert out.shape == g.shape
+    lib().dblp_oracle_sgd_apply(_p(out), _p(g), C.c_float(lr), C.c_uint64(out.size))
+    return out

@@ -52,7 +52,7 @@ EXPORTS = ("dblp_plan_create", "dblp_plan_destroy", "dblp_plan_query", "dblp_pla
            "dblp_apply_loss_resend", "dblp_missing_bits", "dblp_stop_workspace_bytes", "dblp_aggregate_book_stop",
            "dblp_round_until_stop",
            "dblp_aggregate_book",
-           "dblp_aggregate_reduce", "dblp_aggregate", "dblp_round_reset", "dblp_check_bound", "dblp_bound_ok", "dblp_clr",
+           "dblp_aggregate_reduce", "dblp_aggregate_reduce_ex", "dblp_norm_scratch_count", "dblp_aggregate", "dblp_round_reset", "dblp_check_bound", "dblp_bound_ok", "dblp_clr",
            "dblp_select_bound", "dblp_round_host", "dblp_strerror", "dblp_last_error", "dblp_launch_count")
 
 
@@ -247,6 +247,19 @@ def dblp_aggregate_book(plan, hdr_ring, n_slots, arrival, n_arrived_dev, arrival
 def dblp_aggregate_reduce(plan, payload_ring, slot_key, agg_out, flags=DBLP_SUM, stream=None):
     _check(lib().dblp_aggregate_reduce(plan.handle, _ptr(payload_ring), _ptr(slot_key), _ptr(agg_out),
                                        C.c_uint32(flags), _stream(stream)), "dblp_aggregate_reduce")
+
+
+def dblp_norm_scratch_count(plan):
+    n = C.c_uint64()
+    _check(lib().dblp_norm_scratch_count(plan.handle, C.byref(n)), "dblp_norm_scratch_count")
+    return int(n.value)
+
+
+def dblp_aggregate_reduce_ex(plan, payload_ring, slot_key, agg_out, flags=DBLP_SUM, norm_scratch=None, norm_out=None,
+                             params=None, lr=0.0, stream=None):
+    _check(lib().dblp_aggregate_reduce_ex(plan.handle, _ptr(payload_ring), _ptr(slot_key), _ptr(agg_out),
+                                          C.c_uint32(flags), _ptr(norm_scratch), _ptr(norm_out), _ptr(params),
+                                          C.c_float(lr), _stream(stream)), "dblp_aggregate_reduce_ex")
 
 
 def dblp_aggregate(plan, hdr_ring, payload_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, recv_bitmap,

@@ -423,13 +423,24 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-template <int ES, int WB, int J>
-__global__ void __launch_bounds__(kTileThreads, (J == 1 ? DBLP_REDUCE_MIN_BLOCKS : 1))
+// Optional work fused behind the sum (both off in the plain reduce):
+//   norm_partials  one fp64 per tile: the sum of squares of the tile's aggregate values (Eq. 1 needs ||G||); squares of
+//                  fp32 values are exact in fp64, the additions follow a fixed tree (thread, warp shuffle, warps in order)
+//   params / lr    the worker-side update of Algorithm 4, w <- w - lr * g, one fp32 multiply then one fp32 subtract
+struct ReduceExtras {
+    double* norm_partials;
+    float* params;
+    float lr;
+};
+
+template <int ES, int WB, int J, bool EXTRA>
+__global__ void __launch_bounds__(kTileThreads, (J == 1 ? (EXTRA ? DBLP_REDUCE_MIN_BLOCKS - 1 : DBLP_REDUCE_MIN_BLOCKS) : 1))
 k_reduce_tiled(const uint8_t* __restrict__ ring, const unsigned long long* __restrict__ slot_key,
                const uint64_t* __restrict__ chunk_desc, float* __restrict__ agg, uint32_t W, uint32_t C, uint32_t P,
-               uint32_t VPC, uint32_t CH, uint32_t n_tiles, int mean, float Wf)
+               uint32_t VPC, uint32_t CH, uint32_t n_tiles, int mean, float Wf, ReduceExtras ex)
 {
     constexpr int VE = 16 / ES;
+    __shared__ double s_norm[kTileThreads / 32];
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint64_t* sdesc = reinterpret_cast<uint64_t*>(smem_raw);              // [2][CH]
     uint32_t* sslot = reinterpret_cast<uint32_t*>(sdesc + 2 * CH);        // [2][CH][W]
@@ -459,6 +470,7 @@ k_reduce_tiled(const uint8_t* __restrict__ ring, const unsigned long long* __res
         const uint32_t c0 = tile * CH, nch = min(CH, C - c0), nvec = nch * VPC;
         const uint64_t* td = sdesc + buf * CH;
         const uint32_t* ts = sslot + (size_t)buf * CH * W;
+        double sq = 0.0;                      // this thread's share of the tile's sum of squares
         for (uint32_t i0 = tid; i0 < nvec; i0 += kTileThreads * J) {
             float acc[J][VE];
             uint32_t cl[J], v[J], len[J];
@@ -529,26 +541,90 @@ k_reduce_tiled(const uint8_t* __restrict__ ring, const unsigned long long* __res
                     for (int e = 0; e < VE; ++e)
                         if (e < (int)nv) out[e] = acc[j][e];
                 }
+                if (EXTRA) {
+                    if (ex.norm_partials) {
+#pragma unroll
+                        for (int e = 0; e < VE; ++e)
+                            if (e < (int)nv) sq = __dadd_rn(sq, __dmul_rn((double)acc[j][e], (double)acc[j][e]));
+                    }
+                    if (ex.params) {
+                        float* w_out = ex.params + dst[j] + e0;
+#pragma unroll
+                        for (int e = 0; e < VE; ++e)
+                            if (e < (int)nv) w_out[e] = __fsub_rn(w_out[e], __fmul_rn(ex.lr, acc[j][e]));
+                    }
+                }
             }
         }
+        if (EXTRA && ex.norm_partials) {
+#pragma unroll
+            for (int d = 16; d >= 1; d >>= 1) sq = __dadd_rn(sq, __shfl_xor_sync(0xFFFFFFFFu, sq, d));
+            if ((tid & 31) == 0) s_norm[tid >> 5] = sq;
+        }
         __syncthreads();                      // the buffer is refilled by the prefetch of the next iteration
+        if (EXTRA && ex.norm_partials && tid == 0) {
+            double t = 0.0;
+            for (int k = 0; k < kTileThreads / 32; ++k) t = __dadd_rn(t, s_norm[k]);
+            ex.norm_partials[tile] = t;
+        }
     }
     cp_async_wait<0>();
 }
 
+// Sums the per-tile partials in a fixed order (thread t takes t, t + 1024, ...; then a shuffle tree; then the warps in
+// order) and takes the root: out[0] = sum of squares, out[1] = its square root (IEEE).
+__global__ void __launch_bounds__(1024)
+k_norm_finish(const double* __restrict__ partials, uint32_t n, double* __restrict__ out)
+{
+    __shared__ double s_warp[32];
+    double t = 0.0;
+    for (uint32_t k = threadIdx.x; k < n; k += 1024) t = __dadd_rn(t, partials[k]);
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) t = __dadd_rn(t, __shfl_xor_sync(0xFFFFFFFFu, t, d));
+    if ((threadIdx.x & 31) == 0) s_warp[threadIdx.x >> 5] = t;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double all = 0.0;
+        for (int k = 0; k < 32; ++k) all = __dadd_rn(all, s_warp[k]);
+        out[0] = all;
+        out[1] = sqrt(all);
+    }
+}
+
 template <int ES, int WB, int J>
 static cudaError_t launch_tiled(const dblp_plan* p, const uint8_t* ring, const unsigned long long* slot_key, float* agg,
-                                int mean, cudaStream_t s)
+                                int mean, const ReduceExtras* ex, cudaStream_t s)
 {
-    k_reduce_tiled<ES, WB, J><<<p->red_grid, kTileThreads, p->red_smem, s>>>(
-        ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->P, p->VPC, p->red_CH, p->red_tiles, mean, (float)p->W);
+    if (ex)
+        k_reduce_tiled<ES, WB, J, true><<<p->red_grid, kTileThreads, p->red_smem, s>>>(
+            ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->P, p->VPC, p->red_CH, p->red_tiles, mean,
+            (float)p->W, *ex);
+    else
+        k_reduce_tiled<ES, WB, J, false><<<p->red_grid, kTileThreads, p->red_smem, s>>>(
+            ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->P, p->VPC, p->red_CH, p->red_tiles, mean,
+            (float)p->W, ReduceExtras{nullptr, nullptr, 0.0f});
     return cudaGetLastError();
 }
 
 template <int ES, int WB, int J>
 static cudaError_t occupancy_tiled(int* blocks, size_t smem)
 {
-    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, k_reduce_tiled<ES, WB, J>, kTileThreads, smem);
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks, k_reduce_tiled<ES, WB, J, false>, kTileThreads, smem);
+}
+
+static void launch_tiled_for(const dblp_plan* plan, const uint8_t* ring, const unsigned long long* keys, float* agg_out,
+                             int mean, const ReduceExtras* ex, cudaStream_t s)
+{
+    const int J = plan->red_variant;
+    if (plan->es == 4) {
+        if (J == 4) launch_tiled<4, 2, 4>(plan, ring, keys, agg_out, mean, ex, s);
+        else if (J == 2 && plan->W <= 4) launch_tiled<4, 4, 2>(plan, ring, keys, agg_out, mean, ex, s);
+        else launch_tiled<4, 8, kJWide>(plan, ring, keys, agg_out, mean, ex, s);
+    } else {
+        if (J == 4) launch_tiled<2, 2, 4>(plan, ring, keys, agg_out, mean, ex, s);
+        else if (J == 2 && plan->W <= 4) launch_tiled<2, 4, 2>(plan, ring, keys, agg_out, mean, ex, s);
+        else launch_tiled<2, 8, kJWide>(plan, ring, keys, agg_out, mean, ex, s);
+    }
 }
 
 // Chooses the reduce kernel's shape for a plan: worker batch WB and items J so that WB * J = 8 loads are in flight per
@@ -689,16 +765,7 @@ extern "C" int dblp_aggregate_reduce(const dblp_plan_t* plan, const void* payloa
     const uint8_t* ring = static_cast<const uint8_t*>(payload_ring);
     const unsigned long long* keys = reinterpret_cast<const unsigned long long*>(slot_key);
     if (plan->red_variant) {
-        const int J = plan->red_variant;
-        if (plan->es == 4) {
-            if (J == 4) launch_tiled<4, 2, 4>(plan, ring, keys, agg_out, mean, s);
-            else if (J == 2 && plan->W <= 4) launch_tiled<4, 4, 2>(plan, ring, keys, agg_out, mean, s);
-            else launch_tiled<4, 8, kJWide>(plan, ring, keys, agg_out, mean, s);
-        } else {
-            if (J == 4) launch_tiled<2, 2, 4>(plan, ring, keys, agg_out, mean, s);
-            else if (J == 2 && plan->W <= 4) launch_tiled<2, 4, 2>(plan, ring, keys, agg_out, mean, s);
-            else launch_tiled<2, 8, kJWide>(plan, ring, keys, agg_out, mean, s);
-        }
+        launch_tiled_for(plan, ring, keys, agg_out, mean, nullptr, s);
         DBLP_LAUNCHED();
         return DBLP_OK;
     }
@@ -712,6 +779,38 @@ extern "C" int dblp_aggregate_reduce(const dblp_plan_t* plan, const void* payloa
         k_reduce<2><<<(unsigned)grid, kReduceThreads, 0, s>>>(ring, keys, plan->d_chunk_desc, agg_out, plan->W,
                                                               (uint32_t)plan->C, plan->P, plan->VPC, mean, (float)plan->W);
     DBLP_LAUNCHED();
+    return DBLP_OK;
+}
+
+extern "C" int dblp_norm_scratch_count(const dblp_plan_t* plan, uint64_t* count)
+{
+    DBLP_REQUIRE(plan && count, DBLP_EINVAL, "norm_scratch_count: null argument");
+    *count = plan->red_variant ? plan->red_tiles : 0;
+    return DBLP_OK;
+}
+
+extern "C" int dblp_aggregate_reduce_ex(const dblp_plan_t* plan, const void* payload_ring, const uint64_t* slot_key,
+                                        float* agg_out, uint32_t flags, double* norm_scratch, double* norm_out,
+                                        float* params, float lr, void* stream)
+{
+    DBLP_REQUIRE(plan && payload_ring && slot_key && agg_out, DBLP_EINVAL, "aggregate_reduce_ex: null argument");
+    DBLP_REQUIRE(aligned16(payload_ring), DBLP_EALIGN, "aggregate_reduce_ex: payload ring must be 16-byte aligned");
+    DBLP_REQUIRE((reinterpret_cast<uintptr_t>(agg_out) & 3u) == 0 && (reinterpret_cast<uintptr_t>(params) & 3u) == 0 &&
+                 (reinterpret_cast<uintptr_t>(norm_scratch) & 7u) == 0 && (reinterpret_cast<uintptr_t>(norm_out) & 7u) == 0,
+                 DBLP_EALIGN, "aggregate_reduce_ex: misaligned output");
+    DBLP_REQUIRE(flags == DBLP_SUM || flags == DBLP_MEAN, DBLP_EINVAL, "aggregate_reduce_ex: unknown flags %u", flags);
+    DBLP_REQUIRE((norm_scratch == nullptr) == (norm_out == nullptr), DBLP_EINVAL,
+                 "aggregate_reduce_ex: norm_scratch and norm_out go together");
+    DBLP_REQUIRE(plan->red_variant, DBLP_ECAPACITY, "aggregate_reduce_ex: not available for this many workers");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const ReduceExtras ex{norm_scratch, params, lr};
+    launch_tiled_for(plan, static_cast<const uint8_t*>(payload_ring), reinterpret_cast<const unsigned long long*>(slot_key),
+                     agg_out, flags == DBLP_MEAN, &ex, s);
+    DBLP_LAUNCHED();
+    if (norm_scratch) {
+        k_norm_finish<<<1, 1024, 0, s>>>(norm_scratch, plan->red_tiles, norm_out);
+        DBLP_LAUNCHED();
+    }
     return DBLP_OK;
 }
 

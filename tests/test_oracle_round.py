@@ -133,3 +133,36 @@ def test_round_gives_up_after_max_attempts():
     p = orc.Plan([256 * 100], 4, 1024, 2)
     st, attempts, ok, _ = p.round_until_stop(p.headers(1), orc.loss_model("iid", t_drop=TWO32), 1, 1, 8000, 4, False)
     assert attempts == 4 and ok == 0 and popcount(st["bitmap"]) == 0
+
+
+# ------------------------------------------------------------------------------------------------ norm and update
+def test_norm_is_the_exactly_rounded_sum_of_squares():
+    rng = np.random.default_rng(0)
+    for n, scale in ((1, 1.0), (7, 1e-3), (100003, 1e-3), (1 << 20, 1e-4), (50000, 1e10)):
+        g = (rng.standard_normal(n) * scale).astype(np.float32)
+        exact = math.fsum((g.astype(np.float64) ** 2).tolist())         # correctly rounded sum of the exact squares
+        s, nrm = orc.norm(g)
+        assert abs(s - exact) <= 2 * np.spacing(exact)
+        assert nrm == math.sqrt(s)
+    assert orc.norm(np.array([3.0, 4.0], np.float32)) == (25.0, 5.0)
+    assert orc.norm(np.ones(4096, np.float32)) == (4096.0, 64.0)
+    assert orc.norm(np.zeros(10, np.float32)) == (0.0, 0.0)
+    g = (rng.standard_normal(1000) * 1e-3).astype(np.float32)
+    assert orc.norm(2 * g)[0] == 4 * orc.norm(g)[0]                     # scaling by two is exact
+    # a sum where naive accumulation loses the small terms: one large value and a million small ones
+    g = np.concatenate([[4096.0], np.full(1 << 20, 2.0 ** -12)]).astype(np.float32)
+    assert orc.norm(g)[0] == 4096.0 ** 2 + (1 << 20) * 2.0 ** -24
+
+
+def test_sgd_apply_is_multiply_then_subtract_in_fp32():
+    rng = np.random.default_rng(1)
+    w = rng.standard_normal(100000).astype(np.float32)
+    g = (rng.standard_normal(100000) * 1e-3).astype(np.float32)
+    lr = np.float32(0.1)
+    out = orc.sgd_apply(w, g, float(lr))
+    two_step = w - (lr * g)                                              # numpy: two separately rounded fp32 operations
+    assert out.tobytes() == two_step.tobytes()
+    fused = (w.astype(np.float64) - np.float64(lr) * g.astype(np.float64)).astype(np.float32)
+    assert (out != fused).any()                                          # it is NOT the fused multiply-add result
+    assert orc.sgd_apply(w, g, 0.0).tobytes() == w.tobytes()
+    assert orc.sgd_apply(w, np.zeros_like(g), 0.5).tobytes() == w.tobytes()   # lost chunks (zero-filled) change nothing
