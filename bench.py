@@ -256,6 +256,37 @@ def run_gpu(args):
             row["attempt_ratio"] = row["p_low"]["attempts"] / max(1, row["p_high"]["attempts"])
             round_loop.append(row)
 
+    # the reduce with its fused extras (norm for Eq. 1, worker update), timed alone; not part of the timed step
+    extras = None
+    if rank == 0 and world == 1 and not args.no_round_loop:
+        dblp.dblp_round_reset(plan, buf["recv_bitmap"], buf["slot_key"], buf["counters"])
+        step(7)
+        scratch = torch.empty(max(1, dblp.dblp_norm_scratch_count(plan)), dtype=torch.float64, device=dev)
+        norm_out = torch.zeros(2, dtype=torch.float64, device=dev)
+        params = torch.zeros(work.N, dtype=torch.float32, device=dev)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+        def timed(fn, reps=50):
+            for _ in range(3):
+                fn()
+            a.record()
+            for _ in range(reps):
+                fn()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / reps
+
+        extras = {
+            "reduce_ms": timed(lambda: dblp.dblp_aggregate_reduce(plan, buf["payload_ring"], buf["slot_key"], buf["agg"],
+                                                                  dblp.DBLP_MEAN)),
+            "reduce_norm_ms": timed(lambda: dblp.dblp_aggregate_reduce_ex(plan, buf["payload_ring"], buf["slot_key"],
+                                                                          buf["agg"], dblp.DBLP_MEAN, scratch, norm_out)),
+            "reduce_norm_update_ms": timed(lambda: dblp.dblp_aggregate_reduce_ex(
+                plan, buf["payload_ring"], buf["slot_key"], buf["agg"], dblp.DBLP_MEAN, scratch, norm_out, params, 0.01)),
+            "grad_norm": float(norm_out[1].item()),
+        }
+        del scratch, params
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu = cpu_baseline(work, bytes_["total"])
@@ -283,7 +314,7 @@ def run_gpu(args):
         "roofline": {"kernel": "k_reduce", "bound": "hbm", "achieved": red_gbs, "peak": peak, "peak_kind": peak_kind,
                      "unit": "GB/s", "frac": red_gbs / peak, "traffic": TRAFFIC.get(work.name),
                      "algorithmic_bytes_per_launch": bytes_["reduce"], "ms_per_launch": stage_ms["reduce"]},
-        "clocks": clocks, "gpu_launches": launches, "e2e": e2e, "cpu_baseline": cpu, "round_loop": round_loop,
+        "clocks": clocks, "gpu_launches": launches, "e2e": e2e, "cpu_baseline": cpu, "round_loop": round_loop, "reduce_extras": extras,
     }
     print(json.dumps(out))
 

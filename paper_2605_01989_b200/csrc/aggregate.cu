@@ -434,7 +434,7 @@ struct ReduceExtras {
 };
 
 template <int ES, int WB, int J, bool EXTRA>
-__global__ void __launch_bounds__(kTileThreads, (J == 1 ? (EXTRA ? DBLP_REDUCE_MIN_BLOCKS - 1 : DBLP_REDUCE_MIN_BLOCKS) : 1))
+__global__ void __launch_bounds__(kTileThreads, (J == 1 ? DBLP_REDUCE_MIN_BLOCKS : 1))
 k_reduce_tiled(const uint8_t* __restrict__ ring, const unsigned long long* __restrict__ slot_key,
                const uint64_t* __restrict__ chunk_desc, float* __restrict__ agg, uint32_t W, uint32_t C, uint32_t P,
                uint32_t VPC, uint32_t CH, uint32_t n_tiles, int mean, float Wf, ReduceExtras ex)
