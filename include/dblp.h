@@ -43,7 +43,7 @@ typedef enum {
 
 typedef enum { DBLP_F32 = 0, DBLP_BF16 = 1 } dblp_dtype_t;
 typedef enum { DBLP_LOSS_NONE = 0, DBLP_LOSS_IID = 1, DBLP_LOSS_GE = 2, DBLP_LOSS_MICROBURST = 3 } dblp_loss_kind_t;
-enum { DBLP_SUM = 0, DBLP_MEAN = 1 }; /* flags of dblp_aggregate */
+enum { DBLP_SUM = 0, DBLP_MEAN = 1, DBLP_OUT_BF16 = 2 }; /* flags of dblp_aggregate; OUT_BF16 only with dblp_aggregate_reduce_ex */
 
 /* Packet header, 32 bytes, stored beside (not inside) the payload.  seq, round and len_bytes are the paper's
  * three fields (Section IV-A); tensor_id and offset_elems are the id/offset tags of the prior work the paper
@@ -205,6 +205,8 @@ int dblp_aggregate_reduce(const dblp_plan_t* plan, const void* payload_ring, con
  *   update (Algorithm 4, worker: w <- w - alpha * g): params[i] = params[i] - lr * agg[i], an fp32 multiply then an
  *     fp32 subtract (no fused multiply-add), for every element; chunks nobody delivered leave params unchanged because
  *     their aggregate is +0.  params: N fp32, in/out.  NULL = off.
+ *   bf16 output (flag DBLP_OUT_BF16, may be or-ed with DBLP_MEAN): agg_out is N bf16 values, each the fp32 result
+ *     rounded to nearest even (NaN stays a quiet NaN); norm and update still use the fp32 value.
  * For the broadcast half of a round (Algorithm 3 "DBLP_SEND(mean)", Algorithm 4 "DBLP_RECV"), packetize the mean with a
  * W = 1 plan, apply loss, book, and call this with params: the worker's reconstruction and its update in one pass. */
 int dblp_norm_scratch_count(const dblp_plan_t* plan, uint64_t* count);

@@ -595,3 +595,21 @@ void dblp_oracle_sgd_apply(float* params, const float* g, float lr, uint64_t n)
         params[i] = params[i] - step;
     }
 }
+
+/* ---------------------------------------------------------------------------
+ * fp32 -> bf16 with round to nearest, ties to even (the optional 16-bit output
+ * of the aggregate).  bf16 keeps the upper 16 bits of the fp32 pattern; the
+ * discarded 16 bits decide the rounding: above half -> up, below half -> down,
+ * exactly half -> to the even neighbour.  A NaN stays a (quiet) NaN.
+ * ------------------------------------------------------------------------- */
+void dblp_oracle_to_bf16(const float* x, uint16_t* out, uint64_t n)
+{
+    for (uint64_t i = 0; i < n; ++i) {
+        uint32_t b;
+        memcpy(&b, &x[i], 4);
+        uint32_t upper = b >> 16, rest = b & 0xFFFFu;
+        if ((b & 0x7FFFFFFFu) > 0x7F800000u) { out[i] = (uint16_t)(upper | 0x40u); continue; }
+        if (rest > 0x8000u || (rest == 0x8000u && (upper & 1u))) upper += 1;   /* a carry into the exponent is the right result */
+        out[i] = (uint16_t)upper;
+    }
+}

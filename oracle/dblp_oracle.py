@@ -258,3 +258,11 @@ def sgd_apply(params, g, lr):
     assert out.shape == g.shape
     lib().dblp_oracle_sgd_apply(_p(out), _p(g), C.c_float(lr), C.c_uint64(out.size))
     return out
+
+
+def to_bf16(x):
+    """float32 array -> uint16 bf16 patterns, round to nearest even."""
+    x = np.ascontiguousarray(x, np.float32)
+    out = np.empty(x.shape, np.uint16)
+    lib().dblp_oracle_to_bf16(_p(x), _p(out), C.c_uint64(x.size))
+    return out

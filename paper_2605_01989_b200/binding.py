@@ -13,7 +13,7 @@ LIB_PATH = os.path.join(HERE, "libdblp.so")
 
 DBLP_F32, DBLP_BF16 = 0, 1
 DBLP_LOSS_NONE, DBLP_LOSS_IID, DBLP_LOSS_GE, DBLP_LOSS_MICROBURST = 0, 1, 2, 3
-DBLP_SUM, DBLP_MEAN = 0, 1
+DBLP_SUM, DBLP_MEAN, DBLP_OUT_BF16 = 0, 1, 2
 LOSS_KINDS = {"none": DBLP_LOSS_NONE, "iid": DBLP_LOSS_IID, "ge": DBLP_LOSS_GE, "microburst": DBLP_LOSS_MICROBURST}
 HDR_BYTES = 32
 COUNTER_FIELDS = ("n_arrived", "n_accepted", "n_dup", "n_stale", "n_invalid", "n_late")

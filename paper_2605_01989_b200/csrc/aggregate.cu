@@ -427,11 +427,22 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 //   norm_partials  one fp64 per tile: the sum of squares of the tile's aggregate values (Eq. 1 needs ||G||); squares of
 //                  fp32 values are exact in fp64, the additions follow a fixed tree (thread, warp shuffle, warps in order)
 //   params / lr    the worker-side update of Algorithm 4, w <- w - lr * g, one fp32 multiply then one fp32 subtract
+//   out_bf16       the aggregate is stored as bf16 (round to nearest even) instead of fp32; norm and update still use
+//                  the fp32 value
 struct ReduceExtras {
     double* norm_partials;
     float* params;
     float lr;
+    int out_bf16;
 };
+
+// fp32 -> bf16, round to nearest even, NaN kept quiet: the upper 16 bits after adding 0x7FFF plus the lowest kept bit.
+__device__ __forceinline__ uint32_t bf16_rne(float f)
+{
+    const uint32_t b = __float_as_uint(f);
+    if ((b & 0x7FFFFFFFu) > 0x7F800000u) return (b >> 16) | 0x40u;
+    return (b + 0x7FFFu + ((b >> 16) & 1u)) >> 16;
+}
 
 template <int ES, int WB, int J, bool EXTRA>
 __global__ void __launch_bounds__(kTileThreads, (J == 1 ? DBLP_REDUCE_MIN_BLOCKS : 1))
@@ -532,7 +543,20 @@ k_reduce_tiled(const uint8_t* __restrict__ ring, const unsigned long long* __res
                 const uint32_t e0 = v[j] * VE;
                 float* out = agg + dst[j] + e0;
                 const uint32_t nv = min((uint32_t)VE, len[j] - e0);
-                if (nv == VE && (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
+                if (EXTRA && ex.out_bf16) {
+                    uint16_t* out16 = reinterpret_cast<uint16_t*>(agg) + dst[j] + e0;
+                    if (nv == VE && (reinterpret_cast<uintptr_t>(out16) & 7u) == 0) {
+#pragma unroll
+                        for (int q = 0; q < VE / 4; ++q)
+                            reinterpret_cast<uint2*>(out16)[q] =
+                                make_uint2(bf16_rne(acc[j][4 * q]) | (bf16_rne(acc[j][4 * q + 1]) << 16),
+                                           bf16_rne(acc[j][4 * q + 2]) | (bf16_rne(acc[j][4 * q + 3]) << 16));
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < VE; ++e)
+                            if (e < (int)nv) out16[e] = (uint16_t)bf16_rne(acc[j][e]);
+                    }
+                } else if (nv == VE && (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
 #pragma unroll
                     for (int q = 0; q < VE / 4; ++q)
                         st_agg16(out + 4 * q, acc[j][4 * q], acc[j][4 * q + 1], acc[j][4 * q + 2], acc[j][4 * q + 3]);
@@ -602,7 +626,7 @@ static cudaError_t launch_tiled(const dblp_plan* p, const uint8_t* ring, const u
     else
         k_reduce_tiled<ES, WB, J, false><<<p->red_grid, kTileThreads, p->red_smem, s>>>(
             ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->P, p->VPC, p->red_CH, p->red_tiles, mean,
-            (float)p->W, ReduceExtras{nullptr, nullptr, 0.0f});
+            (float)p->W, ReduceExtras{nullptr, nullptr, 0.0f, 0});
     return cudaGetLastError();
 }
 
@@ -795,17 +819,19 @@ extern "C" int dblp_aggregate_reduce_ex(const dblp_plan_t* plan, const void* pay
 {
     DBLP_REQUIRE(plan && payload_ring && slot_key && agg_out, DBLP_EINVAL, "aggregate_reduce_ex: null argument");
     DBLP_REQUIRE(aligned16(payload_ring), DBLP_EALIGN, "aggregate_reduce_ex: payload ring must be 16-byte aligned");
-    DBLP_REQUIRE((reinterpret_cast<uintptr_t>(agg_out) & 3u) == 0 && (reinterpret_cast<uintptr_t>(params) & 3u) == 0 &&
+    DBLP_REQUIRE((reinterpret_cast<uintptr_t>(agg_out) & 1u) == 0 &&
+                 ((flags & DBLP_OUT_BF16) || (reinterpret_cast<uintptr_t>(agg_out) & 3u) == 0) &&
+                 (reinterpret_cast<uintptr_t>(params) & 3u) == 0 &&
                  (reinterpret_cast<uintptr_t>(norm_scratch) & 7u) == 0 && (reinterpret_cast<uintptr_t>(norm_out) & 7u) == 0,
                  DBLP_EALIGN, "aggregate_reduce_ex: misaligned output");
-    DBLP_REQUIRE(flags == DBLP_SUM || flags == DBLP_MEAN, DBLP_EINVAL, "aggregate_reduce_ex: unknown flags %u", flags);
+    DBLP_REQUIRE((flags & ~(uint32_t)(DBLP_MEAN | DBLP_OUT_BF16)) == 0, DBLP_EINVAL, "aggregate_reduce_ex: unknown flags %u", flags);
     DBLP_REQUIRE((norm_scratch == nullptr) == (norm_out == nullptr), DBLP_EINVAL,
                  "aggregate_reduce_ex: norm_scratch and norm_out go together");
     DBLP_REQUIRE(plan->red_variant, DBLP_ECAPACITY, "aggregate_reduce_ex: not available for this many workers");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const ReduceExtras ex{norm_scratch, params, lr};
+    const ReduceExtras ex{norm_scratch, params, lr, (flags & DBLP_OUT_BF16) ? 1 : 0};
     launch_tiled_for(plan, static_cast<const uint8_t*>(payload_ring), reinterpret_cast<const unsigned long long*>(slot_key),
-                     agg_out, flags == DBLP_MEAN, &ex, s);
+                     agg_out, (flags & DBLP_MEAN) ? 1 : 0, &ex, s);
     DBLP_LAUNCHED();
     if (norm_scratch) {
         k_norm_finish<<<1, 1024, 0, s>>>(norm_scratch, plan->red_tiles, norm_out);

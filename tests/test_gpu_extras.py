@@ -72,6 +72,25 @@ def test_fused_norm_and_update(dtype, P, W, flags):
     g.close()
 
 
+@pytest.mark.parametrize("dtype,P,W", [("f32", 1408, 5), ("bf16", 4096, 3), ("f32", 1024, 2)])
+def test_bf16_output_is_the_rounded_fp32_aggregate(dtype, P, W):
+    w = wl.Workload("t", W, dtype, P, RAGGED, 1e-3, wl.LossSpec("iid", 0.1), seed=W + 40, round=2)
+    g, op, o_pay, st = _round(w)
+    out16 = torch.full((op.N + 3,), 0x1234, dtype=torch.int16, device=H.DEV)
+    scratch = torch.empty(dblp.dblp_norm_scratch_count(g.plan), dtype=torch.float64, device=H.DEV)
+    norm = torch.zeros(2, dtype=torch.float64, device=H.DEV)
+    for view in (out16[:op.N], out16[1:op.N + 1]):                   # second view: only 2-byte aligned
+        view.fill_(0x1234)
+        dblp.dblp_aggregate_reduce_ex(g.plan, g.buf["payload_ring"], g.buf["slot_key"], view,
+                                      dblp.DBLP_MEAN | dblp.DBLP_OUT_BF16, scratch, norm)
+        agg = op.reduce(o_pay, st, mean=True)
+        H.assert_bits_equal(view.cpu().numpy().view(np.uint16), orc.to_bf16(agg), "bf16 aggregate")
+        s, _ = orc.norm(agg)
+        assert abs(norm[0].item() - s) <= NORM_RTOL * s                 # the norm is taken before the rounding
+    assert int(out16[op.N + 1].item()) == 0x1234                        # nothing written past the end
+    g.close()
+
+
 def test_norm_of_an_all_lost_round_is_zero():
     w = wl.Workload("t", 3, "f32", 1408, RAGGED, 1e-3, wl.LossSpec("iid", 1.0), seed=1, round=1)
     g, op, o_pay, st = _round(w)

@@ -75,6 +75,21 @@ def test_sweep_points_small():
         H.full_round_parity(p, flags_list=(dblp.DBLP_SUM,))
 
 
+def test_sweep_sample_across_every_axis():
+    """A stride through the cartesian sweep (sizes x workers x payloads x loss rates x processes x seeds), limited to
+    points whose rings the host can hold: every value of every axis occurs at least once."""
+    pts = [p for p in wl.sweep(max_device_bytes=600e6)]
+    sample = pts[::19]
+    assert len(sample) >= 30
+    for axis in ("W", "payload_bytes", "seed"):
+        assert {getattr(p, axis) for p in sample} == {getattr(p, axis) for p in pts}
+    assert {p.loss.kind for p in sample} >= {"none", "iid", "ge"}
+    assert {p.loss.mean_loss for p in sample} >= {0.0, 0.01, 0.05, 0.2}
+    assert len({p.N for p in sample}) >= 4
+    for p in sample:
+        H.full_round_parity(p, flags_list=(dblp.DBLP_MEAN,))
+
+
 def test_stale_duplicate_and_invalid_packets_and_second_attempt():
     w = work(RAGGED, "f32", 1408, 4, wl.LossSpec("iid", 0.3), 21)
     rnd = w.round

@@ -166,3 +166,19 @@ def test_sgd_apply_is_multiply_then_subtract_in_fp32():
     assert (out != fused).any()                                          # it is NOT the fused multiply-add result
     assert orc.sgd_apply(w, g, 0.0).tobytes() == w.tobytes()
     assert orc.sgd_apply(w, np.zeros_like(g), 0.5).tobytes() == w.tobytes()   # lost chunks (zero-filled) change nothing
+
+
+def test_bf16_rounding_matches_the_library_conversion():
+    import torch
+    rng = np.random.default_rng(2)
+    x = np.concatenate([(rng.standard_normal(200000) * 1e-3).astype(np.float32),
+                        rng.integers(0, 1 << 32, 200000, dtype=np.uint64).astype(np.uint32).view(np.float32),
+                        np.array([0.0, -0.0, 1.0, np.inf, -np.inf, 3.3895314e38, 1.00390625, 1.01171875, 1e-40],
+                                 np.float32)])
+    got = orc.to_bf16(x)
+    lib = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    finite = ~np.isnan(x)
+    assert np.array_equal(got[finite], lib[finite])
+    assert ((got[~finite] & 0x7F80) == 0x7F80).all() and ((got[~finite] & 0x7F) != 0).all()     # NaN stays NaN
+    # ties go to the even neighbour: 1 + 2^-8 is halfway between 1.0 (even) and 1 + 2^-7; 1 + 3*2^-8 rounds up to even
+    assert orc.to_bf16(np.array([1.00390625, 1.01171875], np.float32)).tolist() == [0x3F80, 0x3F82]
