@@ -283,6 +283,8 @@ def run_gpu(args):
                                                                           buf["agg"], dblp.DBLP_MEAN, scratch, norm_out)),
             "reduce_norm_update_ms": timed(lambda: dblp.dblp_aggregate_reduce_ex(
                 plan, buf["payload_ring"], buf["slot_key"], buf["agg"], dblp.DBLP_MEAN, scratch, norm_out, params, 0.01)),
+            "reduce_atomic_order_free_ms": timed(lambda: dblp.dblp_aggregate_reduce_atomic(
+                plan, buf["payload_ring"], buf["slot_key"], buf["agg"], dblp.DBLP_MEAN)),
             "grad_norm": float(norm_out[1].item()),
         }
         del scratch, params

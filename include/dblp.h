@@ -214,6 +214,14 @@ int dblp_aggregate_reduce_ex(const dblp_plan_t* plan, const void* payload_ring, 
                              uint32_t flags, double* norm_scratch, double* norm_out, float* params, float lr,
                              void* stream);
 
+/* ---- order-free reduce (property 1: "gradients should be applied as soon as they arrive") --------------------------
+ * Same inputs and the same mathematical result as dblp_aggregate_reduce, but every received payload is added into the
+ * aggregate with floating-point atomics in whatever order the hardware runs them, so the fp32 sums are not
+ * reproducible bit for bit: each element is within (W - 1) * 2^-24 * sum_w |x_w| of the exact sum.  Provided to measure
+ * what the fixed worker order costs; zeroes agg_out first, and scales by 1 / W in a second pass for DBLP_MEAN. */
+int dblp_aggregate_reduce_atomic(const dblp_plan_t* plan, const void* payload_ring, const uint64_t* slot_key,
+                                 float* agg_out, uint32_t flags, void* stream);
+
 /* ---- bookkeeping with early stop (Algorithm 2, the branch without a probe: "if the loss-tolerance threshold is
  * satisfied, send stop") ------------------------------------------------------------------------------------------
  * As dblp_aggregate_book, but each worker's receiver stops the moment its own missing / C <= bound_ppm / 10^6 holds

@@ -52,7 +52,7 @@ EXPORTS = ("dblp_plan_create", "dblp_plan_destroy", "dblp_plan_query", "dblp_pla
            "dblp_apply_loss_resend", "dblp_missing_bits", "dblp_stop_workspace_bytes", "dblp_aggregate_book_stop",
            "dblp_round_until_stop",
            "dblp_aggregate_book",
-           "dblp_aggregate_reduce", "dblp_aggregate_reduce_ex", "dblp_norm_scratch_count", "dblp_aggregate", "dblp_round_reset", "dblp_check_bound", "dblp_bound_ok", "dblp_clr",
+           "dblp_aggregate_reduce", "dblp_aggregate_reduce_ex", "dblp_aggregate_reduce_atomic", "dblp_norm_scratch_count", "dblp_aggregate", "dblp_round_reset", "dblp_check_bound", "dblp_bound_ok", "dblp_clr",
            "dblp_select_bound", "dblp_round_host", "dblp_strerror", "dblp_last_error", "dblp_launch_count")
 
 
@@ -247,6 +247,11 @@ def dblp_aggregate_book(plan, hdr_ring, n_slots, arrival, n_arrived_dev, arrival
 def dblp_aggregate_reduce(plan, payload_ring, slot_key, agg_out, flags=DBLP_SUM, stream=None):
     _check(lib().dblp_aggregate_reduce(plan.handle, _ptr(payload_ring), _ptr(slot_key), _ptr(agg_out),
                                        C.c_uint32(flags), _stream(stream)), "dblp_aggregate_reduce")
+
+
+def dblp_aggregate_reduce_atomic(plan, payload_ring, slot_key, agg_out, flags=DBLP_SUM, stream=None):
+    _check(lib().dblp_aggregate_reduce_atomic(plan.handle, _ptr(payload_ring), _ptr(slot_key), _ptr(agg_out),
+                                              C.c_uint32(flags), _stream(stream)), "dblp_aggregate_reduce_atomic")
 
 
 def dblp_norm_scratch_count(plan):

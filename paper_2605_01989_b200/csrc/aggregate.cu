@@ -848,6 +848,93 @@ extern "C" int dblp_plan_tune_reduce(dblp_plan_t* plan, uint32_t chunks_per_tile
     return rc;
 }
 
+// ------------------------------------------------------------------------------------------------ order-free reduce
+// The alternative the paper's property 1 literally describes ("gradients should be applied as soon as they arrive"):
+// every received payload is added into the aggregate with floating-point atomics, in whatever order the hardware
+// schedules them.  The sum is then not reproducible bit for bit (fp32 addition is not associative); it exists to
+// measure what the fixed worker order of k_reduce_tiled costs.  One thread per (worker, chunk, 16-byte vector).
+namespace dblp {
+
+__device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, float d)
+{
+    asm volatile("red.global.add.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
+template <int ES>
+__global__ void __launch_bounds__(256)
+k_reduce_atomic(const uint8_t* __restrict__ ring, const unsigned long long* __restrict__ slot_key,
+                const uint64_t* __restrict__ chunk_desc, float* __restrict__ agg, uint32_t C, uint32_t P, uint32_t VPC)
+{
+    constexpr int VE = 16 / ES;
+    const uint32_t w = blockIdx.y;
+    const uint64_t i = (uint64_t)blockIdx.x * 256 + threadIdx.x;
+    if (i >= (uint64_t)C * VPC) return;
+    const uint32_t c = (uint32_t)(i / VPC), v = (uint32_t)(i - (uint64_t)c * VPC);
+    const uint32_t slot = reinterpret_cast<const uint2*>(slot_key)[(uint64_t)w * C + c].x;
+    if (slot == kEmpty32) return;
+    const uint64_t d = __ldg(&chunk_desc[c]);
+    const uint32_t len = (uint32_t)(d & 0xFFFFu), e0 = v * VE;
+    if (e0 >= len) return;
+    const uint4 x = ld_payload16(ring + (uint64_t)slot * P + (uint64_t)v * 16);
+    float f[VE];
+    if (ES == 4) {
+        f[0] = __uint_as_float(x.x); f[1] = __uint_as_float(x.y); f[2] = __uint_as_float(x.z); f[3] = __uint_as_float(x.w);
+    } else {
+        const uint32_t wd[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            f[2 * q] = __uint_as_float(wd[q] << 16);
+            f[2 * q + 1] = __uint_as_float(wd[q] & 0xFFFF0000u);
+        }
+    }
+    float* out = agg + (d >> 16) + e0;
+    const uint32_t nv = min((uint32_t)VE, len - e0);
+    if (nv == VE && (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
+#pragma unroll
+        for (int q = 0; q < VE / 4; ++q) red_add_v4(out + 4 * q, f[4 * q], f[4 * q + 1], f[4 * q + 2], f[4 * q + 3]);
+    } else {
+#pragma unroll
+        for (int e = 0; e < VE; ++e)
+            if (e < (int)nv) atomicAdd(out + e, f[e]);
+    }
+}
+
+__global__ void __launch_bounds__(256)
+k_scale(float* __restrict__ agg, uint64_t n, float Wf)
+{
+    const uint64_t i = (uint64_t)blockIdx.x * 256 + threadIdx.x;
+    if (i < n) agg[i] = __fdiv_rn(agg[i], Wf);
+}
+
+}  // namespace dblp
+
+extern "C" int dblp_aggregate_reduce_atomic(const dblp_plan_t* plan, const void* payload_ring, const uint64_t* slot_key,
+                                            float* agg_out, uint32_t flags, void* stream)
+{
+    DBLP_REQUIRE(plan && payload_ring && slot_key && agg_out, DBLP_EINVAL, "aggregate_reduce_atomic: null argument");
+    DBLP_REQUIRE(aligned16(payload_ring), DBLP_EALIGN, "aggregate_reduce_atomic: payload ring must be 16-byte aligned");
+    DBLP_REQUIRE((reinterpret_cast<uintptr_t>(agg_out) & 3u) == 0, DBLP_EALIGN, "aggregate_reduce_atomic: aggregate must be 4-byte aligned");
+    DBLP_REQUIRE(flags == DBLP_SUM || flags == DBLP_MEAN, DBLP_EINVAL, "aggregate_reduce_atomic: unknown flags %u", flags);
+    DBLP_REQUIRE(plan->W <= 65535, DBLP_ECAPACITY, "aggregate_reduce_atomic: more than 65535 workers");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    DBLP_CUDA(cudaMemsetAsync(agg_out, 0, plan->N * sizeof(float), s));          // +0.0f everywhere: lost chunks stay zero
+    const uint64_t gx = (plan->C * plan->VPC + 255) / 256;
+    DBLP_REQUIRE(gx < (1ull << 31), DBLP_ECAPACITY, "aggregate_reduce_atomic: grid too large");
+    dim3 grid((unsigned)gx, plan->W);
+    const uint8_t* ring = static_cast<const uint8_t*>(payload_ring);
+    const unsigned long long* keys = reinterpret_cast<const unsigned long long*>(slot_key);
+    if (plan->es == 4)
+        k_reduce_atomic<4><<<grid, 256, 0, s>>>(ring, keys, plan->d_chunk_desc, agg_out, (uint32_t)plan->C, plan->P, plan->VPC);
+    else
+        k_reduce_atomic<2><<<grid, 256, 0, s>>>(ring, keys, plan->d_chunk_desc, agg_out, (uint32_t)plan->C, plan->P, plan->VPC);
+    DBLP_LAUNCHED();
+    if (flags == DBLP_MEAN) {
+        k_scale<<<(unsigned)((plan->N + 255) / 256), 256, 0, s>>>(agg_out, plan->N, (float)plan->W);
+        DBLP_LAUNCHED();
+    }
+    return DBLP_OK;
+}
+
 extern "C" int dblp_aggregate(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, const void* payload_ring,
                               uint64_t n_slots, const uint32_t* arrival, const uint64_t* n_arrived_dev,
                               uint64_t arrival_cap, uint32_t round, uint32_t* recv_bitmap, uint64_t* slot_key,

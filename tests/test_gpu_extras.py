@@ -91,6 +91,38 @@ def test_bf16_output_is_the_rounded_fp32_aggregate(dtype, P, W):
     g.close()
 
 
+@pytest.mark.parametrize("dtype,P,W", [("f32", 1408, 5), ("bf16", 4096, 3), ("f32", 1024, 32)])
+@pytest.mark.parametrize("flags", [dblp.DBLP_SUM, dblp.DBLP_MEAN])
+def test_order_free_reduce_is_within_the_rounding_bound(dtype, P, W, flags):
+    """Any order of W fp32 additions is within (W-1) * 2^-24 * sum|x| of the exact sum, so the atomic result and the
+    oracle's fixed-order result differ by at most twice that (the mean's division adds one more rounding)."""
+    w = wl.Workload("t", W, dtype, P, RAGGED, 1e-3, wl.LossSpec("iid", 0.15), seed=W + 60, round=2)
+    g, op, o_pay, st = _round(w)
+    dblp.dblp_aggregate_reduce_atomic(g.plan, g.buf["payload_ring"], g.buf["slot_key"], g.buf["agg"], flags)
+    got = g.buf["agg"].cpu().numpy().astype(np.float64)
+    ref = op.reduce(o_pay, st, mean=(flags == dblp.DBLP_MEAN)).astype(np.float64)
+    # sum over the workers that delivered of |x_w|, per element, from the oracle's own packets
+    pay = o_pay.reshape(op.M, op.P)
+    if dtype == "f32":
+        vals = np.abs(pay.view(np.float32).astype(np.float64))
+    else:
+        vals = np.abs(torch.from_numpy(pay.view(np.int16).copy()).view(torch.bfloat16).to(torch.float64).numpy())
+    E = op.E
+    mag = np.zeros(op.N)
+    recv = st["slot_of"].reshape(op.W, op.C) != orc.NONE
+    for t in range(op.T):
+        n, b, c0 = int(op.numel[t]), int(op.base[t]), int(op.chunkbase[t])
+        nch = -(-n // E)
+        for wk in range(op.W):
+            rows = vals[wk * op.C + c0: wk * op.C + c0 + nch] * recv[wk, c0:c0 + nch, None]
+            mag[b:b + n] += rows.reshape(-1)[:n]
+    scale = 1.0 / W if flags == dblp.DBLP_MEAN else 1.0
+    bound = (2 * (W - 1) + 2) * 2.0 ** -24 * mag * scale + 1e-45
+    assert (np.abs(got - ref) <= bound).all()
+    assert (got[mag == 0] == 0).all()                                   # chunks nobody delivered are exactly zero
+    g.close()
+
+
 def test_norm_of_an_all_lost_round_is_zero():
     w = wl.Workload("t", 3, "f32", 1408, RAGGED, 1e-3, wl.LossSpec("iid", 1.0), seed=1, round=1)
     g, op, o_pay, st = _round(w)
