@@ -104,6 +104,12 @@ int dblp_plan_destroy(dblp_plan_t* plan);
 /* C = chunks per worker, N = elements per worker, M = W * C, row_words = ceil(C / 32) words per bitmap row.
  * Any out pointer may be NULL. */
 int dblp_plan_query(const dblp_plan_t* plan, uint64_t* C, uint64_t* N, uint64_t* M, uint64_t* row_words);
+/* Where packets live.  DBLP_WIRE_RINGS (default): a header ring of 32-byte entries and a payload ring of payload_bytes
+ * entries.  DBLP_WIRE_DATAGRAMS: one ring of (32 + payload_bytes)-byte datagrams, header first, as a packet looks on
+ * the wire (Section IV-B: chunk and header together fill the UDP payload); pass the ring's base as both hdr_ring and
+ * payload_ring to every call.  Set before the first round; results do not depend on it. */
+enum { DBLP_WIRE_RINGS = 0, DBLP_WIRE_DATAGRAMS = 1 };
+int dblp_plan_set_wire_format(dblp_plan_t* plan, int format);
 /* Expert knob: pins the launch shape of the masked reduce (dblp_aggregate_reduce) -- chunks summed per tile and
  * number of persistent blocks; 0 = choose automatically (what dblp_plan_create does).  Results do not depend on it.
  * DBLP_ECAPACITY if the tile's slot entries do not fit in shared memory.  Not to be called while work that uses the

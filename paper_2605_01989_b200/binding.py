@@ -47,7 +47,8 @@ class DblpError(RuntimeError):
 
 
 _lib = None
-EXPORTS = ("dblp_plan_create", "dblp_plan_destroy", "dblp_plan_query", "dblp_plan_tune_reduce", "dblp_workspace_bytes",
+EXPORTS = ("dblp_plan_create", "dblp_plan_destroy", "dblp_plan_query", "dblp_plan_tune_reduce", "dblp_plan_set_wire_format",
+           "dblp_workspace_bytes",
            "dblp_loss_model_from_rates", "dblp_packetize", "dblp_apply_loss", "dblp_apply_loss_static",
            "dblp_apply_loss_resend", "dblp_missing_bits", "dblp_stop_workspace_bytes", "dblp_aggregate_book_stop",
            "dblp_round_until_stop",
@@ -134,6 +135,11 @@ class Plan:
         ws = C.c_size_t()
         _check(lib().dblp_workspace_bytes(self.handle, C.byref(ws)), "dblp_workspace_bytes")
         self.workspace_bytes = int(ws.value)
+
+    def set_wire_format(self, datagrams):
+        """True: one ring of (32 + P)-byte datagrams (pass it as both hdr_ring and payload_ring); False: two rings."""
+        _check(lib().dblp_plan_set_wire_format(self.handle, C.c_int(1 if datagrams else 0)), "dblp_plan_set_wire_format")
+        self.datagrams = bool(datagrams)
 
     def tune_reduce(self, chunks_per_tile=0, grid_blocks=0):
         _check(lib().dblp_plan_tune_reduce(self.handle, C.c_uint32(chunks_per_tile), C.c_uint32(grid_blocks)),

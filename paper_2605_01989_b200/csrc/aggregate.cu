@@ -26,7 +26,7 @@ k_book(const dblp_hdr_t* __restrict__ hdr_ring, uint64_t n_slots, const uint32_t
        const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap, uint32_t round,
        unsigned long long* __restrict__ slot_key, dblp_counters_t* counters,
        const uint64_t* __restrict__ numel, const uint32_t* __restrict__ chunkbase,
-       uint32_t T, uint32_t W, uint64_t C, uint32_t E, uint32_t es)
+       uint32_t T, uint32_t W, uint64_t C, uint32_t E, uint32_t es, uint32_t hdr_stride)
 {
     const uint64_t n = min(*n_arrived_dev, arrival_cap);
     const uint64_t a = (uint64_t)blockIdx.x * kBookThreads + threadIdx.x;
@@ -38,7 +38,7 @@ k_book(const dblp_hdr_t* __restrict__ hdr_ring, uint64_t n_slots, const uint32_t
         bool valid = false;
         uint4 h0 = make_uint4(0, 0, 0, 0), h1 = h0;
         if (slot < n_slots) {
-            const uint4* hp = reinterpret_cast<const uint4*>(hdr_ring + slot);
+            const uint4* hp = reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(hdr_ring) + (uint64_t)slot * hdr_stride);
             h0 = __ldg(hp);       // seq, round, len_bytes, tensor_id
             h1 = __ldg(hp + 1);   // offset lo, offset hi, worker, reserved
             const uint64_t off = (uint64_t)h1.x | ((uint64_t)h1.y << 32);
@@ -122,7 +122,7 @@ k_book_claim(const dblp_hdr_t* __restrict__ hdr_ring, uint64_t n_slots, const ui
              const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap, uint32_t round,
              unsigned long long* __restrict__ slot_key, dblp_counters_t* counters, uint32_t* __restrict__ cell_of,
              const uint64_t* __restrict__ numel, const uint32_t* __restrict__ chunkbase,
-             uint32_t T, uint32_t W, uint64_t C, uint32_t E, uint32_t es)
+             uint32_t T, uint32_t W, uint64_t C, uint32_t E, uint32_t es, uint32_t hdr_stride)
 {
     const uint64_t n = min(*n_arrived_dev, arrival_cap);
     const uint64_t a = (uint64_t)blockIdx.x * kBookThreads + threadIdx.x;
@@ -134,7 +134,7 @@ k_book_claim(const dblp_hdr_t* __restrict__ hdr_ring, uint64_t n_slots, const ui
         bool valid = false;
         uint4 h0 = make_uint4(0, 0, 0, 0), h1 = h0;
         if (slot < n_slots) {
-            const uint4* hp = reinterpret_cast<const uint4*>(hdr_ring + slot);
+            const uint4* hp = reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(hdr_ring) + (uint64_t)slot * hdr_stride);
             h0 = __ldg(hp);
             h1 = __ldg(hp + 1);
             const uint64_t off = (uint64_t)h1.x | ((uint64_t)h1.y << 32);
@@ -621,11 +621,11 @@ static cudaError_t launch_tiled(const dblp_plan* p, const uint8_t* ring, const u
 {
     if (ex)
         k_reduce_tiled<ES, WB, J, true><<<p->red_grid, kTileThreads, p->red_smem, s>>>(
-            ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->P, p->VPC, p->red_CH, p->red_tiles, mean,
+            ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->pay_stride, p->VPC, p->red_CH, p->red_tiles, mean,
             (float)p->W, *ex);
     else
         k_reduce_tiled<ES, WB, J, false><<<p->red_grid, kTileThreads, p->red_smem, s>>>(
-            ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->P, p->VPC, p->red_CH, p->red_tiles, mean,
+            ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->pay_stride, p->VPC, p->red_CH, p->red_tiles, mean,
             (float)p->W, ReduceExtras{nullptr, nullptr, 0.0f, 0});
     return cudaGetLastError();
 }
@@ -713,7 +713,7 @@ extern "C" int dblp_aggregate_book(const dblp_plan_t* plan, const dblp_hdr_t* hd
         const unsigned grid = (unsigned)((arrival_cap + kBookThreads - 1) / kBookThreads);
         k_book<<<grid, kBookThreads, 0, s>>>(hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round,
                                              reinterpret_cast<unsigned long long*>(slot_key), counters, plan->d_numel,
-                                             plan->d_chunkbase, plan->T, plan->W, plan->C, plan->E, plan->es);
+                                             plan->d_chunkbase, plan->T, plan->W, plan->C, plan->E, plan->es, plan->hdr_stride);
         DBLP_LAUNCHED();
     }
     const uint64_t cells = plan->row_words * 32 * plan->W;
@@ -759,7 +759,7 @@ extern "C" int dblp_aggregate_book_stop(const dblp_plan_t* plan, const dblp_hdr_
         const unsigned grid = (unsigned)((arrival_cap + kBookThreads - 1) / kBookThreads);
         k_book_claim<<<grid, kBookThreads, 0, s>>>(hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, keys, counters,
                                                    cell_of, plan->d_numel, plan->d_chunkbase, plan->T, plan->W, plan->C,
-                                                   plan->E, plan->es);
+                                                   plan->E, plan->es, plan->hdr_stride);
         DBLP_LAUNCHED();
         k_stop_count<<<l.n_blocks, 256, plan->W * sizeof(uint32_t), s>>>(cell_of, keys, n_arrived_dev, arrival_cap, counters,
                                                                         plan->W, plan->C, block_cnt);
@@ -786,7 +786,7 @@ extern "C" int dblp_aggregate_reduce(const dblp_plan_t* plan, const void* payloa
     DBLP_REQUIRE(flags == DBLP_SUM || flags == DBLP_MEAN, DBLP_EINVAL, "aggregate_reduce: unknown flags %u", flags);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int mean = flags == DBLP_MEAN;
-    const uint8_t* ring = static_cast<const uint8_t*>(payload_ring);
+    const uint8_t* ring = static_cast<const uint8_t*>(payload_ring) + plan->pay_off;
     const unsigned long long* keys = reinterpret_cast<const unsigned long long*>(slot_key);
     if (plan->red_variant) {
         launch_tiled_for(plan, ring, keys, agg_out, mean, nullptr, s);
@@ -798,10 +798,10 @@ extern "C" int dblp_aggregate_reduce(const dblp_plan_t* plan, const void* payloa
     DBLP_REQUIRE(grid < (1ull << 31), DBLP_ECAPACITY, "aggregate_reduce: grid too large");
     if (plan->es == 4)
         k_reduce<4><<<(unsigned)grid, kReduceThreads, 0, s>>>(ring, keys, plan->d_chunk_desc, agg_out, plan->W,
-                                                              (uint32_t)plan->C, plan->P, plan->VPC, mean, (float)plan->W);
+                                                              (uint32_t)plan->C, plan->pay_stride, plan->VPC, mean, (float)plan->W);
     else
         k_reduce<2><<<(unsigned)grid, kReduceThreads, 0, s>>>(ring, keys, plan->d_chunk_desc, agg_out, plan->W,
-                                                              (uint32_t)plan->C, plan->P, plan->VPC, mean, (float)plan->W);
+                                                              (uint32_t)plan->C, plan->pay_stride, plan->VPC, mean, (float)plan->W);
     DBLP_LAUNCHED();
     return DBLP_OK;
 }
@@ -830,7 +830,7 @@ extern "C" int dblp_aggregate_reduce_ex(const dblp_plan_t* plan, const void* pay
     DBLP_REQUIRE(plan->red_variant, DBLP_ECAPACITY, "aggregate_reduce_ex: not available for this many workers");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const ReduceExtras ex{norm_scratch, params, lr, (flags & DBLP_OUT_BF16) ? 1 : 0};
-    launch_tiled_for(plan, static_cast<const uint8_t*>(payload_ring), reinterpret_cast<const unsigned long long*>(slot_key),
+    launch_tiled_for(plan, static_cast<const uint8_t*>(payload_ring) + plan->pay_off, reinterpret_cast<const unsigned long long*>(slot_key),
                      agg_out, (flags & DBLP_MEAN) ? 1 : 0, &ex, s);
     DBLP_LAUNCHED();
     if (norm_scratch) {
@@ -921,12 +921,12 @@ extern "C" int dblp_aggregate_reduce_atomic(const dblp_plan_t* plan, const void*
     const uint64_t gx = (plan->C * plan->VPC + 255) / 256;
     DBLP_REQUIRE(gx < (1ull << 31), DBLP_ECAPACITY, "aggregate_reduce_atomic: grid too large");
     dim3 grid((unsigned)gx, plan->W);
-    const uint8_t* ring = static_cast<const uint8_t*>(payload_ring);
+    const uint8_t* ring = static_cast<const uint8_t*>(payload_ring) + plan->pay_off;
     const unsigned long long* keys = reinterpret_cast<const unsigned long long*>(slot_key);
     if (plan->es == 4)
-        k_reduce_atomic<4><<<grid, 256, 0, s>>>(ring, keys, plan->d_chunk_desc, agg_out, (uint32_t)plan->C, plan->P, plan->VPC);
+        k_reduce_atomic<4><<<grid, 256, 0, s>>>(ring, keys, plan->d_chunk_desc, agg_out, (uint32_t)plan->C, plan->pay_stride, plan->VPC);
     else
-        k_reduce_atomic<2><<<grid, 256, 0, s>>>(ring, keys, plan->d_chunk_desc, agg_out, (uint32_t)plan->C, plan->P, plan->VPC);
+        k_reduce_atomic<2><<<grid, 256, 0, s>>>(ring, keys, plan->d_chunk_desc, agg_out, (uint32_t)plan->C, plan->pay_stride, plan->VPC);
     DBLP_LAUNCHED();
     if (flags == DBLP_MEAN) {
         k_scale<<<(unsigned)((plan->N + 255) / 256), 256, 0, s>>>(agg_out, plan->N, (float)plan->W);

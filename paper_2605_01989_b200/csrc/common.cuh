@@ -86,6 +86,9 @@ __device__ __forceinline__ uint4 draw(const DrawKey& k, uint64_t a, uint32_t str
 //   bucket_bounds[0..B], bound_ppm[B] (staging for per-bucket tolerances)
 struct dblp_plan {
     uint32_t T, W, B, P, es, E, VE, VPC;
+    // where packets live: header of slot i at hdr_ring + i * hdr_stride, payload at payload_ring + pay_off + i * pay_stride
+    // (separate rings: 32, P, 0; datagrams with the header in front: 32 + P, 32 + P, 32)
+    uint32_t hdr_stride, pay_stride, pay_off;
     int dtype, device;
     uint64_t C, N, M, row_words;
     std::vector<uint64_t> h_numel, h_base;

@@ -3,8 +3,7 @@
 // A pure copy, bound by HBM.  A block owns a tile of CH consecutive chunks of one worker: it first brings the tile's
 // chunk descriptors into shared memory (so that no payload load waits on a table lookup), writes the tile's headers,
 // then streams the tile's 16-byte vectors, kPackUnroll per thread per pass with all loads issued before the first
-// store.  The destination of a tile is one contiguous stretch of the ring; the source follows the descriptors, so
-// tensors of any size are handled: a vector that is ragged (end of a short chunk) or whose source is not 16-byte
+// store.  The source follows the descriptors, so tensors of any size are handled: a vector that is ragged (end of a short chunk) or whose source is not 16-byte
 // aligned is assembled from element loads, and the slot's tail is written as zero.
 #include "common.cuh"
 
@@ -35,7 +34,8 @@ constexpr uint32_t kPackMaxTile = 256;     // chunks per tile at most (descripto
 
 template <int ES>
 __global__ void __launch_bounds__(kPackThreads)
-k_packetize(GradPtrs grads, uint32_t w0, uint32_t C, uint32_t VPC, uint32_t P, uint32_t CH, uint32_t round,
+k_packetize(GradPtrs grads, uint32_t w0, uint32_t C, uint32_t VPC, uint32_t pay_stride, uint32_t hdr_stride, uint32_t CH,
+            uint32_t round,
             const uint64_t* __restrict__ chunk_desc, const uint32_t* __restrict__ chunk_tensor,
             const uint64_t* __restrict__ tensor_base, dblp_hdr_t* __restrict__ hdr_ring, uint8_t* __restrict__ ring)
 {
@@ -51,14 +51,14 @@ k_packetize(GradPtrs grads, uint32_t w0, uint32_t C, uint32_t VPC, uint32_t P, u
         s_desc[k] = d;
         const uint32_t t = __ldg(&chunk_tensor[c0 + k]);
         const uint64_t off = (d >> 16) - __ldg(&tensor_base[t]);
-        uint4* h = reinterpret_cast<uint4*>(hdr_ring + slot0 + k);
+        uint4* h = reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(hdr_ring) + (slot0 + k) * hdr_stride);
         h[0] = make_uint4(c0 + k, round, (uint32_t)(d & 0xFFFFu) * ES, t);
         h[1] = make_uint4((uint32_t)off, (uint32_t)(off >> 32), w, 0u);
     }
     __syncthreads();
 
     const uint32_t nvec = nch * VPC;
-    uint8_t* __restrict__ out = ring + slot0 * P;                 // the tile's slots are contiguous
+    uint8_t* __restrict__ out = ring + slot0 * pay_stride;        // first slot of the tile
     for (uint32_t i0 = tid; i0 < nvec; i0 += kPackThreads * kPackUnroll) {
         uint4 val[kPackUnroll];
 #pragma unroll
@@ -89,7 +89,9 @@ k_packetize(GradPtrs grads, uint32_t w0, uint32_t C, uint32_t VPC, uint32_t P, u
 #pragma unroll
         for (int u = 0; u < kPackUnroll; ++u) {
             const uint32_t i = i0 + u * kPackThreads;
-            if (i < nvec) st_stream16(out + (uint64_t)i * 16, val[u]);
+            if (i >= nvec) continue;
+            const uint32_t cl = i / VPC, v = i - cl * VPC;
+            st_stream16(out + (uint64_t)cl * pay_stride + (uint64_t)v * 16, val[u]);
         }
     }
 }
@@ -119,11 +121,11 @@ extern "C" int dblp_packetize(const dblp_plan_t* plan, const void* const* grads,
         for (uint32_t k = 0; k < nw; ++k) gp.p[k] = grads[w0 + k];
         dim3 grid((unsigned)gx, nw);
         if (plan->es == 4)
-            k_packetize<4><<<grid, kPackThreads, 0, s>>>(gp, w0, (uint32_t)plan->C, plan->VPC, plan->P, CH, round,
-                plan->d_chunk_desc, plan->d_chunk_tensor, plan->d_base, hdr_ring, static_cast<uint8_t*>(payload_ring));
+            k_packetize<4><<<grid, kPackThreads, 0, s>>>(gp, w0, (uint32_t)plan->C, plan->VPC, plan->pay_stride, plan->hdr_stride, CH, round,
+                plan->d_chunk_desc, plan->d_chunk_tensor, plan->d_base, hdr_ring, static_cast<uint8_t*>(payload_ring) + plan->pay_off);
         else
-            k_packetize<2><<<grid, kPackThreads, 0, s>>>(gp, w0, (uint32_t)plan->C, plan->VPC, plan->P, CH, round,
-                plan->d_chunk_desc, plan->d_chunk_tensor, plan->d_base, hdr_ring, static_cast<uint8_t*>(payload_ring));
+            k_packetize<2><<<grid, kPackThreads, 0, s>>>(gp, w0, (uint32_t)plan->C, plan->VPC, plan->pay_stride, plan->hdr_stride, CH, round,
+                plan->d_chunk_desc, plan->d_chunk_tensor, plan->d_base, hdr_ring, static_cast<uint8_t*>(payload_ring) + plan->pay_off);
         DBLP_LAUNCHED();
     }
     return DBLP_OK;

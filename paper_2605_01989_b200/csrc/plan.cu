@@ -61,6 +61,7 @@ extern "C" int dblp_plan_create(const uint64_t* tensor_numel, uint32_t T, int dt
     p->E = payload_bytes / p->es;
     p->VE = 16 / p->es;
     p->VPC = payload_bytes / 16;
+    p->hdr_stride = 32; p->pay_stride = payload_bytes; p->pay_off = 0;
     p->d_numel = p->d_base = nullptr; p->d_chunk_desc = nullptr;
     p->d_chunkbase = p->d_chunk_tensor = p->d_bucket_bounds = p->d_bound_ppm = nullptr;
 
@@ -124,6 +125,19 @@ extern "C" int dblp_plan_create(const uint64_t* tensor_numel, uint32_t T, int dt
         return rc;
     }
     *out = p;
+    return DBLP_OK;
+}
+
+extern "C" int dblp_plan_set_wire_format(dblp_plan_t* plan, int format)
+{
+    DBLP_REQUIRE(plan, DBLP_EINVAL, "plan_set_wire_format: null plan");
+    if (format == DBLP_WIRE_RINGS) {
+        plan->hdr_stride = 32; plan->pay_stride = plan->P; plan->pay_off = 0;
+    } else if (format == DBLP_WIRE_DATAGRAMS) {
+        plan->hdr_stride = plan->pay_stride = 32 + plan->P; plan->pay_off = 32;
+    } else {
+        DBLP_REQUIRE(false, DBLP_EINVAL, "plan_set_wire_format: unknown format %d", format);
+    }
     return DBLP_OK;
 }
 

@@ -193,6 +193,37 @@ def test_physically_permuted_ring():
     g.close()
 
 
+@pytest.mark.parametrize("dtype,P", [("f32", 1408), ("bf16", 4096)])
+def test_datagram_wire_format(dtype, P):
+    """Header and payload interleaved in one ring, as a packet looks on the wire: same results, different addresses."""
+    w = work(RAGGED, dtype, P, 4, wl.LossSpec("ge", 0.1, 5.0), 51)
+    rnd = w.round
+    grads = wl.make_grads(w, H.DEV)
+    op = orc.Plan(w.numel, w.elem_size, P, 4)
+    gm, om = H.models_for(w, op.C)
+    g = H.GpuRound(w)
+    g.plan.set_wire_format(True)
+    b = g.buf
+    ring = torch.full((op.M * (32 + P) + 16,), 0xCD, dtype=torch.uint8, device=H.DEV)
+    dblp.dblp_packetize(g.plan, grads, rnd, ring, ring)
+    o_hdr, o_pay = op.packetize(H.to_host(grads, dtype), rnd)
+    expect = np.concatenate([o_hdr.view(np.uint8).reshape(op.M, 32), o_pay.reshape(op.M, P)], axis=1).reshape(-1)
+    H.assert_bits_equal(ring.cpu().numpy()[:op.M * (32 + P)], expect, "datagram ring")
+    assert bool((ring[op.M * (32 + P):] == 0xCD).all())
+    g.apply_loss(gm, w.seed, rnd)
+    dblp.dblp_aggregate(g.plan, ring, ring, op.M, b["arrival"], b["n_arrived"], op.M, rnd, b["recv_bitmap"], b["slot_key"],
+                        b["counters"], b["agg"], dblp.DBLP_MEAN)
+    o_del, _ = op.loss_mask(om, w.seed, rnd)
+    o_arr, o_n = op.arrival(o_del, w.seed, rnd)
+    st = op.book(o_hdr, o_arr, o_n, rnd, op.new_state())
+    H.compare_state(g, st, op)
+    H.assert_bits_equal(b["agg"].cpu().numpy(), op.reduce(o_pay, st, mean=True), "aggregate from datagrams")
+    dblp.dblp_aggregate_reduce_atomic(g.plan, ring, b["slot_key"], b["agg"], dblp.DBLP_SUM)
+    ref = op.reduce(o_pay, st)
+    assert np.allclose(b["agg"].cpu().numpy(), ref, rtol=0, atol=1e-8)
+    g.close()
+
+
 def test_round_host_entry_point_matches_the_oracle():
     w = work(RAGGED, "f32", 1408, 3, wl.LossSpec("ge", 0.05, 6.0), 41)
     op = orc.Plan(w.numel, 4, 1408, 3)
