@@ -253,7 +253,8 @@ int dblp_round_reset(const dblp_plan_t* plan, uint32_t* recv_bitmap, uint64_t* s
  * For each worker w and bucket b: recv_cnt[w*B+b] = set bits of row w over the bucket's sequence range,
  * missing_cnt = total - recv_cnt, ok = (missing * 10^6 <= bound_ppm * total) in 64-bit integers;
  * *all_ok = 1 iff every ok is 1.  bound_ppm: HOST, n_bounds = 1 (one tolerance for all) or B (per bucket), in parts
- * per million (Table I: 0.8 % = 8000).  Outputs: recv_cnt, missing_cnt u32[W*B], ok u8[W*B], all_ok u32[1]. */
+ * per million (Table I: 0.8 % = 8000).  Outputs: recv_cnt, missing_cnt u32[W*B], ok u8[W*B], all_ok u32[1].
+ * A plan serves one dblp_check_bound at a time (calls on one stream, or ordered by events). */
 int dblp_check_bound(const dblp_plan_t* plan, const uint32_t* recv_bitmap, const uint32_t* bound_ppm,
                      uint32_t n_bounds, uint32_t* recv_cnt, uint32_t* missing_cnt, uint8_t* ok, uint32_t* all_ok,
                      void* stream);

@@ -9,9 +9,10 @@ constexpr int kBoundThreads = 512;
 __global__ void __launch_bounds__(kBoundThreads)
 k_bound(const uint32_t* __restrict__ bitmap, uint64_t row_words, const uint32_t* __restrict__ bucket_bounds, uint32_t B,
         uint32_t bound_scalar, const uint32_t* __restrict__ bound_per_bucket, uint32_t* __restrict__ recv_cnt,
-        uint32_t* __restrict__ missing_cnt, uint8_t* __restrict__ ok)
+        uint32_t* __restrict__ missing_cnt, uint8_t* ok, uint32_t* __restrict__ all_ok, uint32_t* ticket)
 {
     __shared__ uint32_t s_warp[kBoundThreads / 32];
+    __shared__ bool s_last;
     const uint32_t b = blockIdx.x, w = blockIdx.y;
     const uint32_t lo = bucket_bounds[b], hi = bucket_bounds[b + 1];
     const uint32_t* row = bitmap + (uint64_t)w * row_words;
@@ -37,16 +38,21 @@ k_bound(const uint32_t* __restrict__ bitmap, uint64_t row_words, const uint32_t*
         recv_cnt[cell] = got;
         missing_cnt[cell] = (uint32_t)miss;
         ok[cell] = miss * 1000000ull <= p * total;
+        // the block that finishes last (a counter, nobody waits) folds the flags into all_ok and rearms the counter
+        __threadfence();
+        s_last = atomicAdd(ticket, 1u) == gridDim.x * gridDim.y - 1;
     }
-}
-
-__global__ void __launch_bounds__(256)
-k_bound_all(const uint8_t* __restrict__ ok, uint32_t cells, uint32_t* __restrict__ all_ok)
-{
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
     int bad = 0;
-    for (uint32_t i = threadIdx.x; i < cells; i += 256) bad |= !ok[i];
+    const uint32_t cells = gridDim.x * gridDim.y;
+    for (uint32_t i = threadIdx.x; i < cells; i += kBoundThreads) bad |= !__ldcg(&ok[i]);
     const int any_bad = __syncthreads_or(bad);
-    if (threadIdx.x == 0) *all_ok = any_bad ? 0u : 1u;
+    if (threadIdx.x == 0) {
+        *all_ok = any_bad ? 0u : 1u;
+        *ticket = 0;
+    }
 }
 
 }  // namespace dblp
@@ -69,9 +75,7 @@ extern "C" int dblp_check_bound(const dblp_plan_t* plan, const uint32_t* recv_bi
     }
     dim3 grid(plan->B, plan->W);
     k_bound<<<grid, kBoundThreads, 0, s>>>(recv_bitmap, plan->row_words, plan->d_bucket_bounds, plan->B, bound_ppm[0],
-                                           per_bucket, recv_cnt, missing_cnt, ok);
-    DBLP_LAUNCHED();
-    k_bound_all<<<1, 256, 0, s>>>(ok, plan->W * plan->B, all_ok);
+                                           per_bucket, recv_cnt, missing_cnt, ok, all_ok, plan->d_ticket);
     DBLP_LAUNCHED();
     return DBLP_OK;
 }

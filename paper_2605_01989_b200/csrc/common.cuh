@@ -83,7 +83,8 @@ __device__ __forceinline__ uint4 draw(const DrawKey& k, uint64_t a, uint32_t str
 //   chunk_desc[c]   = (first element of chunk c in the flat gradient) << 16 | elements in the chunk
 //   chunk_tensor[c] = tensor the chunk belongs to
 //   numel[t], base[t] (first flat element of tensor t), chunkbase[t] (sequence number of its first chunk; [T] = C)
-//   bucket_bounds[0..B], bound_ppm[B] (staging for per-bucket tolerances)
+//   bucket_bounds[0..B], bound_ppm[B] (staging for per-bucket tolerances), ticket (see k_bound)
+// The staging buffer and the ticket make a plan serve one dblp_check_bound at a time.
 struct dblp_plan {
     uint32_t T, W, B, P, es, E, VE, VPC;
     // where packets live: header of slot i at hdr_ring + i * hdr_stride, payload at payload_ring + pay_off + i * pay_stride
@@ -100,6 +101,7 @@ struct dblp_plan {
     uint32_t* d_chunk_tensor;
     uint32_t* d_bucket_bounds;
     uint32_t* d_bound_ppm;
+    uint32_t* d_ticket;     // "blocks finished" counter of k_bound; zero between launches
     // launch shape of the masked reduce (configure_reduce): red_variant = items per thread of the tiled kernel,
     // 0 = the simple one-vector-per-thread kernel
     uint32_t red_variant, red_CH, red_tiles, red_grid;

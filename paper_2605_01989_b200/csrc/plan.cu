@@ -30,6 +30,7 @@ static void free_tables(dblp_plan* p)
     cudaFree(p->d_chunk_tensor);
     cudaFree(p->d_bucket_bounds);
     cudaFree(p->d_bound_ppm);
+    cudaFree(p->d_ticket);
 }
 
 template <typename T>
@@ -63,7 +64,7 @@ extern "C" int dblp_plan_create(const uint64_t* tensor_numel, uint32_t T, int dt
     p->VPC = payload_bytes / 16;
     p->hdr_stride = 32; p->pay_stride = payload_bytes; p->pay_off = 0;
     p->d_numel = p->d_base = nullptr; p->d_chunk_desc = nullptr;
-    p->d_chunkbase = p->d_chunk_tensor = p->d_bucket_bounds = p->d_bound_ppm = nullptr;
+    p->d_chunkbase = p->d_chunk_tensor = p->d_bucket_bounds = p->d_bound_ppm = p->d_ticket = nullptr;
 
     uint64_t base = 0, c = 0;
     p->h_numel.assign(tensor_numel, tensor_numel + T);
@@ -112,6 +113,8 @@ extern "C" int dblp_plan_create(const uint64_t* tensor_numel, uint32_t T, int dt
     if (e == cudaSuccess) e = upload(&p->d_chunk_tensor, owner);
     if (e == cudaSuccess) e = upload(&p->d_bucket_bounds, bounds);
     if (e == cudaSuccess) e = cudaMalloc((void**)&p->d_bound_ppm, sizeof(uint32_t) * B);
+    if (e == cudaSuccess) e = cudaMalloc((void**)&p->d_ticket, sizeof(uint32_t));
+    if (e == cudaSuccess) e = cudaMemset(p->d_ticket, 0, sizeof(uint32_t));
     if (e != cudaSuccess) {
         set_error("plan: device table setup failed: %s", cudaGetErrorString(e));
         free_tables(p);

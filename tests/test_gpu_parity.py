@@ -294,5 +294,5 @@ def test_library_counts_its_launches():
     g.apply_loss(gm, 1, 1)
     g.aggregate(1)
     g.check_bound(1000)
-    assert dblp.dblp_launch_count() - n0 == 1 + 6 + 3 + 2
+    assert dblp.dblp_launch_count() - n0 == 1 + 6 + 3 + 1
     g.close()
