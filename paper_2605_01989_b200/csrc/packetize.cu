@@ -32,6 +32,17 @@ __device__ __forceinline__ void st_stream16(void* p, uint4 v)
 
 constexpr uint32_t kPackMaxTile = 256;     // chunks per tile at most (descriptors live in static shared memory)
 
+// Headers are re-read in arrival (that is, random) order by the bookkeeping a moment later: ask L2 to keep them
+// while the payloads stream through.
+__device__ __forceinline__ void st_keep16(void* p, uint4 v)
+{
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(policy));
+    asm volatile("st.global.L2::cache_hint.v4.u32 [%0], {%1,%2,%3,%4}, %5;" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w),
+                 "l"(policy)
+                 : "memory");
+}
+
 template <int ES>
 __global__ void __launch_bounds__(kPackThreads)
 k_packetize(GradPtrs grads, uint32_t w0, uint32_t C, uint32_t VPC, uint32_t pay_stride, uint32_t hdr_stride, uint32_t CH,
@@ -52,8 +63,8 @@ k_packetize(GradPtrs grads, uint32_t w0, uint32_t C, uint32_t VPC, uint32_t pay_
         const uint32_t t = __ldg(&chunk_tensor[c0 + k]);
         const uint64_t off = (d >> 16) - __ldg(&tensor_base[t]);
         uint4* h = reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(hdr_ring) + (slot0 + k) * hdr_stride);
-        h[0] = make_uint4(c0 + k, round, (uint32_t)(d & 0xFFFFu) * ES, t);
-        h[1] = make_uint4((uint32_t)off, (uint32_t)(off >> 32), w, 0u);
+        st_keep16(h, make_uint4(c0 + k, round, (uint32_t)(d & 0xFFFFu) * ES, t));
+        st_keep16(h + 1, make_uint4((uint32_t)off, (uint32_t)(off >> 32), w, 0u));
     }
     __syncthreads();
 
