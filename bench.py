@@ -358,6 +358,68 @@ def run_gpu(args):
     print(json.dumps(out))
 
 
+def run_sweep(args):
+    """Stand-alone timing of packetize and of the aggregate path (bookkeeping + reduce + bound check) over the size
+    sweep: per-worker buffer 1 MiB * 4^k, W in {2, 8, 32}, payload {1024, 4096}, 5 % bursty loss.  Points that do not
+    fit in device memory are left out.  Prints one JSON line."""
+    from paper_2605_01989_b200 import binding as dblp
+    torch.cuda.set_device(0)
+    dev = "cuda:0"
+    peak, peak_kind = measured_peak()
+    rows = []
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for k in range(6):
+        for W in (2, 8, 32):
+            for P in (1024, 4096):
+                work = wl.sweep_point((1 << 20) * 4 ** k, W, P, 0.05, "ge", 10)
+                free, _ = torch.cuda.mem_get_info()
+                if work.device_bytes() + (2 << 30) > free:
+                    rows.append({"buffer_MiB": 4 ** k, "W": W, "P": P, "skipped": "does not fit"})
+                    continue
+                plan = dblp.Plan(work.numel, work.dtype, work.payload_bytes, work.W)
+                buf = plan.alloc_round(dev)
+                grads = wl.make_grads(work, dev)
+                model = dblp.loss_model(work.loss.kind, **work.loss.thresholds(plan.C))
+                reps = max(3, min(50, int(2e10 / work.device_bytes())))
+
+                def timed(fn):
+                    for _ in range(2):
+                        fn()
+                    a.record()
+                    for _ in range(reps):
+                        fn()
+                    b.record()
+                    torch.cuda.synchronize()
+                    return a.elapsed_time(b) / reps
+
+                t_pack = timed(lambda: dblp.dblp_packetize(plan, grads, 1, buf["hdr_ring"], buf["payload_ring"]))
+                dblp.dblp_apply_loss(plan, model, work.seed, 1, 0, buf["delivered_bits"], buf["arrival"],
+                                     buf["n_arrived"], buf["ws"])
+
+                def agg_path():
+                    dblp.dblp_round_reset(plan, buf["recv_bitmap"], buf["slot_key"], buf["counters"])
+                    dblp.dblp_aggregate(plan, buf["hdr_ring"], buf["payload_ring"], plan.M, buf["arrival"],
+                                        buf["n_arrived"], plan.M, 1, buf["recv_bitmap"], buf["slot_key"],
+                                        buf["counters"], buf["agg"], dblp.DBLP_MEAN)
+                    dblp.dblp_check_bound(plan, buf["recv_bitmap"], 50000, buf["recv_cnt"], buf["missing_cnt"],
+                                          buf["ok"], buf["all_ok"])
+
+                t_agg = timed(agg_path)
+                t_red = timed(lambda: dblp.dblp_aggregate_reduce(plan, buf["payload_ring"], buf["slot_key"], buf["agg"],
+                                                                 dblp.DBLP_MEAN))
+                n = int(buf["n_arrived"].item())
+                by = byte_model(work, plan.C, n, int(n / plan.M * work.W * work.N * work.elem_size))
+                rows.append({"buffer_MiB": 4 ** k, "W": W, "P": P, "packets": plan.M, "loss": 1 - n / plan.M,
+                             "packetize_GBps": by["packetize"] / t_pack / 1e6,
+                             "aggregate_path_GBps": (by["book"] + by["reduce"] + by["check_bound"]) / t_agg / 1e6,
+                             "reduce_GBps": by["reduce"] / t_red / 1e6, "reduce_frac_of_%s" % peak_kind: by["reduce"] / t_red / 1e6 / peak,
+                             "aggregate_path_us": t_agg * 1e3})
+                plan.close()
+                del buf, grads
+                torch.cuda.empty_cache()
+    print(json.dumps({"sweep": rows, "peak": peak, "peak_kind": peak_kind}))
+
+
 # DRAM bytes (read + write) per k_reduce launch from an ncu capture of this same workload; None until captured, and
 # reset to None whenever the kernel changes.
 TRAFFIC = {"resnet50-f32": 882.8e6}
@@ -463,7 +525,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-round-loop", action="store_true")
     ap.add_argument("--serial", action="store_true", help="all stages on one stream")
+    ap.add_argument("--sweep", action="store_true", help="time the size sweep instead of the default step")
     args = ap.parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     if args.impl == "reference":
         args.steps = 5 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup

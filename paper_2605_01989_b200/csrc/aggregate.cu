@@ -405,6 +405,9 @@ k_reduce(const uint8_t* __restrict__ ring, const unsigned long long* __restrict_
 #ifndef DBLP_REDUCE_MIN_BLOCKS
 #define DBLP_REDUCE_MIN_BLOCKS 4   // caps the one-item variant at 64 registers: four 256-thread blocks per SM
 #endif
+#ifndef DBLP_REDUCE_MIN_BLOCKS_WIDE
+#define DBLP_REDUCE_MIN_BLOCKS_WIDE 3   // resident blocks of the variants that hold 32 accumulators (bf16 with W <= 4, W = 1)
+#endif
 #ifndef DBLP_REDUCE_J_WIDE
 #define DBLP_REDUCE_J_WIDE 1      // items per thread when W > 4 (8 workers per batch)
 #endif
@@ -445,7 +448,7 @@ __device__ __forceinline__ uint32_t bf16_rne(float f)
 }
 
 template <int ES, int WB, int J, bool EXTRA>
-__global__ void __launch_bounds__(kTileThreads, (J == 1 ? DBLP_REDUCE_MIN_BLOCKS : 1))
+__global__ void __launch_bounds__(kTileThreads, ((ES == 4 && J < 8) || J == 1 ? DBLP_REDUCE_MIN_BLOCKS : DBLP_REDUCE_MIN_BLOCKS_WIDE))
 k_reduce_tiled(const uint8_t* __restrict__ ring, const unsigned long long* __restrict__ slot_key,
                const uint64_t* __restrict__ chunk_desc, float* __restrict__ agg, uint32_t W, uint32_t C, uint32_t P,
                uint32_t VPC, uint32_t CH, uint32_t n_tiles, int mean, float Wf, ReduceExtras ex)
@@ -457,6 +460,7 @@ k_reduce_tiled(const uint8_t* __restrict__ ring, const unsigned long long* __res
     uint32_t* sslot = reinterpret_cast<uint32_t*>(sdesc + 2 * CH);        // [2][CH][W]
     const uint32_t tid = threadIdx.x;
     const uint2* cells = reinterpret_cast<const uint2*>(slot_key);
+    const uint32_t vpc_magic = (uint32_t)((0x100000000ull + VPC - 1) / VPC);   // ceil(2^32 / VPC); unused for VPC = 1
 
     auto prefetch = [&](uint32_t tile, uint32_t buf) {
         const uint32_t c0 = tile * CH, nch = min(CH, C - c0);
@@ -491,7 +495,7 @@ k_reduce_tiled(const uint8_t* __restrict__ ring, const unsigned long long* __res
             for (int j = 0; j < J; ++j) {
                 const uint32_t i = i0 + j * kTileThreads;
                 act[j] = i < nvec;
-                cl[j] = act[j] ? i / VPC : 0;
+                cl[j] = !act[j] ? 0 : ((J > 1 && J < 8) || VPC == 1) ? i / VPC : __umulhi(i, vpc_magic);   // i / VPC (exact for i < 2^32 / VPC)
                 v[j] = i - cl[j] * VPC;
                 const uint64_t d = td[cl[j]];
                 len[j] = (uint32_t)(d & 0xFFFFu);
@@ -536,9 +540,12 @@ k_reduce_tiled(const uint8_t* __restrict__ ring, const unsigned long long* __res
 #pragma unroll
             for (int j = 0; j < J; ++j) {
                 if (!act[j]) continue;
-                if (mean) {
+                if (mean == 1) {
 #pragma unroll
                     for (int e = 0; e < VE; ++e) acc[j][e] = __fdiv_rn(acc[j][e], Wf);
+                } else if (mean == 2) {                    // W a power of two: times 1/W is the same rounding, and cheaper
+#pragma unroll
+                    for (int e = 0; e < VE; ++e) acc[j][e] = __fmul_rn(acc[j][e], Wf);
                 }
                 const uint32_t e0 = v[j] * VE;
                 float* out = agg + dst[j] + e0;
@@ -619,14 +626,21 @@ template <int ES, int WB, int J>
 static cudaError_t launch_tiled(const dblp_plan* p, const uint8_t* ring, const unsigned long long* slot_key, float* agg,
                                 int mean, const ReduceExtras* ex, cudaStream_t s)
 {
+    // sum / (float)W: for W = 1 nothing to do, for a power of two a multiplication by the exact reciprocal gives the
+    // identical correctly rounded result, otherwise an IEEE division
+    float Wf = (float)p->W;
+    if (mean) {
+        if (p->W == 1) mean = 0;
+        else if ((p->W & (p->W - 1)) == 0) { mean = 2; Wf = 1.0f / (float)p->W; }
+    }
     if (ex)
         k_reduce_tiled<ES, WB, J, true><<<p->red_grid, kTileThreads, p->red_smem, s>>>(
             ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->pay_stride, p->VPC, p->red_CH, p->red_tiles, mean,
-            (float)p->W, *ex);
+            Wf, *ex);
     else
         k_reduce_tiled<ES, WB, J, false><<<p->red_grid, kTileThreads, p->red_smem, s>>>(
             ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->pay_stride, p->VPC, p->red_CH, p->red_tiles, mean,
-            (float)p->W, ReduceExtras{nullptr, nullptr, 0.0f, 0});
+            Wf, ReduceExtras{nullptr, nullptr, 0.0f, 0});
     return cudaGetLastError();
 }
 
@@ -640,6 +654,11 @@ static void launch_tiled_for(const dblp_plan* plan, const uint8_t* ring, const u
                              int mean, const ReduceExtras* ex, cudaStream_t s)
 {
     const int J = plan->red_variant;
+    if (J == 8) {
+        if (plan->es == 4) launch_tiled<4, 1, 8>(plan, ring, keys, agg_out, mean, ex, s);
+        else launch_tiled<2, 1, 8>(plan, ring, keys, agg_out, mean, ex, s);
+        return;
+    }
     if (plan->es == 4) {
         if (J == 4) launch_tiled<4, 2, 4>(plan, ring, keys, agg_out, mean, ex, s);
         else if (J == 2 && plan->W <= 4) launch_tiled<4, 4, 2>(plan, ring, keys, agg_out, mean, ex, s);
@@ -652,7 +671,7 @@ static void launch_tiled_for(const dblp_plan* plan, const uint8_t* ring, const u
 }
 
 // Chooses the reduce kernel's shape for a plan: worker batch WB and items J so that WB * J = 8 loads are in flight per
-// thread, the tile height CH, and the grid.  Measured on B200 over payloads of 1408 and 4096 bytes, small tiles with one
+// thread (W = 1: 1 x 8, W = 2: 2 x 4, W <= 4: 4 x 2, else 8 x 1), the tile height CH, and the grid.  Measured on B200 over payloads of 1408 and 4096 bytes, small tiles with one
 // block per tile (the hardware hands out tiles as blocks retire) beat one resident wave of persistent blocks by 1-3 %,
 // so that is the default; the persistent loop serves grids capped by the caller.  ch_override / grid_override
 // (0 = automatic) pin the shape.
@@ -660,7 +679,7 @@ int configure_reduce(dblp_plan* p, uint32_t ch_override, uint32_t grid_override)
 {
     p->red_variant = 0;
     const uint32_t W = p->W;
-    const int J = W <= 2 ? 4 : (W <= 4 ? 2 : kJWide);
+    const int J = W == 1 ? 8 : W <= 2 ? 4 : (W <= 4 ? 2 : kJWide);
     // Tile height: eight chunks, or more when chunks are so short that eight would not give every thread two items.
     uint32_t CH = 8;
     const uint32_t want = (2u * kTileThreads * J + p->VPC - 1) / p->VPC;
@@ -669,8 +688,10 @@ int configure_reduce(dblp_plan* p, uint32_t ch_override, uint32_t grid_override)
     const size_t smem_cap = 48 * 1024;
     if (per_chunk > smem_cap) return DBLP_OK;              // slot entries of one chunk do not fit: simple kernel
     if (CH * per_chunk > smem_cap) CH = (uint32_t)(smem_cap / per_chunk);
+    const uint64_t ch_div_cap = 0x100000000ull / ((uint64_t)p->VPC * p->VPC);   // keeps the kernel's multiply-high division exact
+    if (CH > ch_div_cap) CH = (uint32_t)ch_div_cap;
     if (ch_override) {
-        if (ch_override * per_chunk > smem_cap) return DBLP_ECAPACITY;
+        if (ch_override * per_chunk > smem_cap || ch_override > ch_div_cap) return DBLP_ECAPACITY;
         CH = ch_override;
     }
     if (CH > p->C) CH = (uint32_t)p->C;
@@ -680,7 +701,8 @@ int configure_reduce(dblp_plan* p, uint32_t ch_override, uint32_t grid_override)
     int sms = 0, blocks = 0;
     cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, p->device);
     if (e == cudaSuccess) {
-        if (p->es == 4) e = J == 4 ? occupancy_tiled<4, 2, 4>(&blocks, p->red_smem) : (J == 2 && W <= 4) ? occupancy_tiled<4, 4, 2>(&blocks, p->red_smem) : occupancy_tiled<4, 8, kJWide>(&blocks, p->red_smem);
+        if (J == 8) e = p->es == 4 ? occupancy_tiled<4, 1, 8>(&blocks, p->red_smem) : occupancy_tiled<2, 1, 8>(&blocks, p->red_smem);
+        else if (p->es == 4) e = J == 4 ? occupancy_tiled<4, 2, 4>(&blocks, p->red_smem) : (J == 2 && W <= 4) ? occupancy_tiled<4, 4, 2>(&blocks, p->red_smem) : occupancy_tiled<4, 8, kJWide>(&blocks, p->red_smem);
         else            e = J == 4 ? occupancy_tiled<2, 2, 4>(&blocks, p->red_smem) : (J == 2 && W <= 4) ? occupancy_tiled<2, 4, 2>(&blocks, p->red_smem) : occupancy_tiled<2, 8, kJWide>(&blocks, p->red_smem);
     }
     if (e != cudaSuccess) { set_error("reduce set-up failed: %s", cudaGetErrorString(e)); return DBLP_ECUDA; }
