@@ -602,6 +602,163 @@ k_reduce_tiled(const uint8_t* __restrict__ ring, const unsigned long long* __res
     cp_async_wait<0>();
 }
 
+// ------------------------------------------------------------------------------------------------ warp-per-chunk reduce
+// Same tiles, same tables in shared memory, same arithmetic as k_reduce_tiled, but a warp owns a whole chunk: its
+// descriptor and its W slot entries are read once per chunk (they are the same for all lanes), lane l handles the
+// vectors l, l + 32, ... of the chunk, S of them at a time, so that WB * S = 8 payload loads are in flight per thread
+// with almost no index arithmetic per load.
+template <int ES, int WB, int S, bool EXTRA>
+__global__ void __launch_bounds__(kTileThreads, (S == 1 || (ES == 4 && S < 8)) ? DBLP_REDUCE_MIN_BLOCKS : DBLP_REDUCE_MIN_BLOCKS_WIDE)
+k_reduce_rows(const uint8_t* __restrict__ ring, const unsigned long long* __restrict__ slot_key,
+              const uint64_t* __restrict__ chunk_desc, float* __restrict__ agg, uint32_t W, uint32_t C, uint32_t P,
+              uint32_t CH, uint32_t n_tiles, int mean, float Wf, ReduceExtras ex)
+{
+    constexpr int VE = 16 / ES;
+    constexpr uint32_t kWarps = kTileThreads / 32;
+    __shared__ double s_norm[kWarps];
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint64_t* sdesc = reinterpret_cast<uint64_t*>(smem_raw);              // [2][CH]
+    uint32_t* sslot = reinterpret_cast<uint32_t*>(sdesc + 2 * CH);        // [2][CH][W]
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint2* cells = reinterpret_cast<const uint2*>(slot_key);
+
+    auto prefetch = [&](uint32_t tile, uint32_t buf) {
+        const uint32_t c0 = tile * CH, nch = min(CH, C - c0);
+        uint32_t* dst = sslot + (size_t)buf * CH * W;
+        for (uint32_t k = tid; k < nch * W; k += kTileThreads) {
+            const uint32_t w = k / nch, cl = k - w * nch;
+            cp_async4(&dst[cl * W + w], &cells[(uint64_t)w * C + c0 + cl].x);
+        }
+        for (uint32_t k = tid; k < nch; k += kTileThreads) cp_async8(&sdesc[buf * CH + k], &chunk_desc[c0 + k]);
+    };
+
+    uint32_t tile = blockIdx.x, buf = 0;
+    if (tile < n_tiles) prefetch(tile, 0);
+    cp_async_commit();
+    for (; tile < n_tiles; tile += gridDim.x, buf ^= 1) {
+        const uint32_t next = tile + gridDim.x;
+        if (next < n_tiles) prefetch(next, buf ^ 1);
+        cp_async_commit();
+        cp_async_wait<1>();
+        __syncthreads();
+
+        const uint32_t nch = min(CH, C - tile * CH);
+        const uint64_t* td = sdesc + buf * CH;
+        const uint32_t* ts = sslot + (size_t)buf * CH * W;
+        double sq = 0.0;
+        for (uint32_t cl = warp; cl < nch; cl += kWarps) {
+            const uint64_t d = td[cl];
+            const uint32_t len = (uint32_t)(d & 0xFFFFu);
+            const uint32_t nvc = (len + VE - 1) / VE;                    // vectors that hold data
+            float* const out_row = agg + (d >> 16);
+            for (uint32_t vb = 0; vb < nvc; vb += 32 * S) {
+                float acc[S][VE];
+#pragma unroll
+                for (int s = 0; s < S; ++s)
+#pragma unroll
+                    for (int e = 0; e < VE; ++e) acc[s][e] = 0.0f;
+                for (uint32_t wb = 0; wb < W; wb += WB) {
+                    uint32_t slot[WB];
+                    uint4 x[S][WB];
+#pragma unroll
+                    for (int k = 0; k < WB; ++k) slot[k] = (wb + k < W) ? ts[cl * W + wb + k] : kEmpty32;
+#pragma unroll
+                    for (int k = 0; k < WB; ++k) {
+                        if (slot[k] == kEmpty32) continue;             // the same for the whole warp
+                        const uint8_t* src = ring + (uint64_t)slot[k] * P + (uint64_t)(vb + lane) * 16;
+#pragma unroll
+                        for (int s = 0; s < S; ++s)
+                            if (vb + lane + 32 * s < nvc) x[s][k] = ld_payload16(src + 512 * s);
+                    }
+#pragma unroll
+                    for (int k = 0; k < WB; ++k) {                      // worker order: the additions are not reassociated
+                        if (slot[k] == kEmpty32) continue;
+#pragma unroll
+                        for (int s = 0; s < S; ++s) {
+                            if (vb + lane + 32 * s >= nvc) continue;
+                            if (ES == 4) {
+                                acc[s][0] = __fadd_rn(acc[s][0], __uint_as_float(x[s][k].x));
+                                acc[s][1] = __fadd_rn(acc[s][1], __uint_as_float(x[s][k].y));
+                                acc[s][2] = __fadd_rn(acc[s][2], __uint_as_float(x[s][k].z));
+                                acc[s][3] = __fadd_rn(acc[s][3], __uint_as_float(x[s][k].w));
+                            } else {
+                                const uint32_t wd[4] = {x[s][k].x, x[s][k].y, x[s][k].z, x[s][k].w};
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    acc[s][2 * q] = __fadd_rn(acc[s][2 * q], __uint_as_float(wd[q] << 16));
+                                    acc[s][2 * q + 1] = __fadd_rn(acc[s][2 * q + 1], __uint_as_float(wd[q] & 0xFFFF0000u));
+                                }
+                            }
+                        }
+                    }
+                }
+#pragma unroll
+                for (int s = 0; s < S; ++s) {
+                    const uint32_t v = vb + lane + 32 * s;
+                    if (v >= nvc) continue;
+                    if (mean == 1) {
+#pragma unroll
+                        for (int e = 0; e < VE; ++e) acc[s][e] = __fdiv_rn(acc[s][e], Wf);
+                    } else if (mean == 2) {                // W a power of two: times 1/W is the same rounding, and cheaper
+#pragma unroll
+                        for (int e = 0; e < VE; ++e) acc[s][e] = __fmul_rn(acc[s][e], Wf);
+                    }
+                    const uint32_t e0 = v * VE;
+                    float* out = out_row + e0;
+                    const uint32_t nv = min((uint32_t)VE, len - e0);
+                    if (EXTRA && ex.out_bf16) {
+                        uint16_t* out16 = reinterpret_cast<uint16_t*>(agg) + (d >> 16) + e0;
+                        if (nv == VE && (reinterpret_cast<uintptr_t>(out16) & 7u) == 0) {
+#pragma unroll
+                            for (int q = 0; q < VE / 4; ++q)
+                                reinterpret_cast<uint2*>(out16)[q] =
+                                    make_uint2(bf16_rne(acc[s][4 * q]) | (bf16_rne(acc[s][4 * q + 1]) << 16),
+                                               bf16_rne(acc[s][4 * q + 2]) | (bf16_rne(acc[s][4 * q + 3]) << 16));
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < VE; ++e)
+                                if (e < (int)nv) out16[e] = (uint16_t)bf16_rne(acc[s][e]);
+                        }
+                    } else if (nv == VE && (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
+#pragma unroll
+                        for (int q = 0; q < VE / 4; ++q)
+                            st_agg16(out + 4 * q, acc[s][4 * q], acc[s][4 * q + 1], acc[s][4 * q + 2], acc[s][4 * q + 3]);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < VE; ++e)
+                            if (e < (int)nv) out[e] = acc[s][e];
+                    }
+                    if (EXTRA) {
+                        if (ex.norm_partials) {
+#pragma unroll
+                            for (int e = 0; e < VE; ++e)
+                                if (e < (int)nv) sq = __dadd_rn(sq, __dmul_rn((double)acc[s][e], (double)acc[s][e]));
+                        }
+                        if (ex.params) {
+                            float* w_out = ex.params + (d >> 16) + e0;
+#pragma unroll
+                            for (int e = 0; e < VE; ++e)
+                                if (e < (int)nv) w_out[e] = __fsub_rn(w_out[e], __fmul_rn(ex.lr, acc[s][e]));
+                        }
+                    }
+                }
+            }
+        }
+        if (EXTRA && ex.norm_partials) {
+#pragma unroll
+            for (int dlt = 16; dlt >= 1; dlt >>= 1) sq = __dadd_rn(sq, __shfl_xor_sync(0xFFFFFFFFu, sq, dlt));
+            if (lane == 0) s_norm[warp] = sq;
+        }
+        __syncthreads();
+        if (EXTRA && ex.norm_partials && tid == 0) {
+            double t = 0.0;
+            for (uint32_t k = 0; k < kWarps; ++k) t = __dadd_rn(t, s_norm[k]);
+            ex.norm_partials[tile] = t;
+        }
+    }
+    cp_async_wait<0>();
+}
+
 // Sums the per-tile partials in a fixed order (thread t takes t, t + 1024, ...; then a shuffle tree; then the warps in
 // order) and takes the root: out[0] = sum of squares, out[1] = its square root (IEEE).
 __global__ void __launch_bounds__(1024)
@@ -632,6 +789,17 @@ static cudaError_t launch_tiled(const dblp_plan* p, const uint8_t* ring, const u
     if (mean) {
         if (p->W == 1) mean = 0;
         else if ((p->W & (p->W - 1)) == 0) { mean = 2; Wf = 1.0f / (float)p->W; }
+    }
+    if (p->red_rows) {
+        if (ex)
+            k_reduce_rows<ES, WB, J, true><<<p->red_grid, kTileThreads, p->red_smem, s>>>(
+                ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->pay_stride, p->red_CH, p->red_tiles, mean, Wf,
+                *ex);
+        else
+            k_reduce_rows<ES, WB, J, false><<<p->red_grid, kTileThreads, p->red_smem, s>>>(
+                ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->pay_stride, p->red_CH, p->red_tiles, mean, Wf,
+                ReduceExtras{nullptr, nullptr, 0.0f, 0});
+        return cudaGetLastError();
     }
     if (ex)
         k_reduce_tiled<ES, WB, J, true><<<p->red_grid, kTileThreads, p->red_smem, s>>>(
@@ -679,6 +847,9 @@ int configure_reduce(dblp_plan* p, uint32_t ch_override, uint32_t grid_override)
 {
     p->red_variant = 0;
     const uint32_t W = p->W;
+    // Few workers and long payloads: the warp-per-chunk kernel (one table lookup per chunk instead of per vector) is
+    // 20-50 % faster there (measured: W = 1, 2 at 4096-byte payloads); elsewhere the per-vector kernel is 2-3 % ahead.
+    p->red_rows = (W <= 4 && p->VPC >= 128) ? 1 : 0;
     const int J = W == 1 ? 8 : W <= 2 ? 4 : (W <= 4 ? 2 : kJWide);
     // Tile height: eight chunks, or more when chunks are so short that eight would not give every thread two items.
     uint32_t CH = 8;

@@ -104,7 +104,7 @@ struct dblp_plan {
     uint32_t* d_ticket;     // "blocks finished" counter of k_bound; zero between launches
     // launch shape of the masked reduce (configure_reduce): red_variant = items per thread of the tiled kernel,
     // 0 = the simple one-vector-per-thread kernel
-    uint32_t red_variant, red_CH, red_tiles, red_grid;
+    uint32_t red_variant, red_CH, red_tiles, red_grid, red_rows;
     size_t red_smem;
 };
 

@@ -36,7 +36,8 @@ def _round(w):
     return g, op, o_pay, st
 
 
-@pytest.mark.parametrize("dtype,P,W", [("f32", 1408, 5), ("bf16", 4096, 3), ("f32", 1024, 2), ("f32", 4096, 17)])
+@pytest.mark.parametrize("dtype,P,W", [("f32", 1408, 5), ("bf16", 4096, 3), ("f32", 1024, 2), ("f32", 4096, 17),
+                                       ("f32", 4096, 1), ("bf16", 2048, 2)])
 @pytest.mark.parametrize("flags", [dblp.DBLP_SUM, dblp.DBLP_MEAN])
 def test_fused_norm_and_update(dtype, P, W, flags):
     w = wl.Workload("t", W, dtype, P, RAGGED, 1e-3, wl.LossSpec("ge", 0.1, 5.0), seed=W, round=4)

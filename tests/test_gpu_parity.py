@@ -36,6 +36,15 @@ def test_worker_counts(W):
     H.full_round_parity(work(ALIGNED, "f32", 1024, W, wl.LossSpec("iid", 0.2), 5))
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("P", [2048, 4096, 65536])
+@pytest.mark.parametrize("W", [1, 2, 3, 4])
+def test_few_workers_long_payloads(W, P, dtype):
+    """The shape that takes the warp-per-chunk reduce kernel: ragged tensors, short last chunks, unaligned bases."""
+    numel = [100003, 1, 4096, 5, 16384 * 3 + 7, 31, 2048]
+    H.full_round_parity(work(numel, dtype, P, W, wl.LossSpec("iid", 0.2), 70 + W))
+
+
 def test_total_loss_and_zero_loss():
     r = H.full_round_parity(work(RAGGED, "f32", 1408, 3, wl.LossSpec("iid", 1.0), 2))
     assert r["n_arrived"] == 0
