@@ -6,12 +6,14 @@
 //           minimum on the claimed cell.  Integer atomics only, so every result is independent of thread order.
 // k_bitmap  warp ballot over the cells of a row -> one bitmap word per warp; also folds this call's arrival count
 //           into the counters (after every k_book thread has read the old value).
-// k_reduce_tiled  the bandwidth-bound kernel (see the comment above it); k_reduce is its simple form, kept for
-//           worker counts whose slot entries do not fit in shared memory.
-// k_reduce  one thread per (chunk, 16-byte vector).  It reads the W cell entries of its
-//           chunk, issues up to eight independent 128-bit streaming loads (one per worker that delivered), adds them
-//           in worker order into fp32 accumulators and writes the aggregate with 128-bit stores.  A worker whose
-//           packet was lost costs no payload traffic.
+// k_reduce_tiled  the bandwidth-bound kernel: one thread per (chunk, 16-byte vector), tables of a tile of chunks
+//           staged in shared memory, eight 128-bit streaming payload loads in flight per thread, fp32 additions in
+//           worker order, 128-bit streaming stores.  A worker whose packet was lost costs no payload traffic.
+// k_reduce_rows   the same with a warp per chunk; chosen for few workers with long payloads.
+// k_reduce  the simple form (tables read from global memory), kept for worker counts whose slot entries do not
+//           fit in shared memory.
+// Further down: bookkeeping with early stop (k_book_claim, k_stop_*), the fp64 norm finish, the order-free atomic
+// reduce kept for comparison.
 #include "common.cuh"
 
 namespace dblp {
