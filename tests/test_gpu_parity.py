@@ -45,6 +45,19 @@ def test_few_workers_long_payloads(W, P, dtype):
     H.full_round_parity(work(numel, dtype, P, W, wl.LossSpec("iid", 0.2), 70 + W))
 
 
+def test_thousands_of_workers_take_the_simple_reduce_kernel():
+    """More workers than one chunk's slot entries fit in shared memory: the reduce falls back to its simple form, the
+    fused extras say so instead of running, packetize goes through its worker groups."""
+    w = work([100, 7, 64], "f32", 64, 6200, wl.LossSpec("iid", 0.3), 5, bounds=(0, 300000, 1000000))
+    H.full_round_parity(w)
+    g = H.GpuRound(w)
+    assert dblp.dblp_norm_scratch_count(g.plan) == 0
+    with pytest.raises(dblp.DblpError) as e:
+        dblp.dblp_aggregate_reduce_ex(g.plan, g.buf["payload_ring"], g.buf["slot_key"], g.buf["agg"], dblp.DBLP_SUM)
+    assert e.value.status == -3
+    g.close()
+
+
 def test_total_loss_and_zero_loss():
     r = H.full_round_parity(work(RAGGED, "f32", 1408, 3, wl.LossSpec("iid", 1.0), 2))
     assert r["n_arrived"] == 0
