@@ -45,6 +45,36 @@ def test_few_workers_long_payloads(W, P, dtype):
     H.full_round_parity(work(numel, dtype, P, W, wl.LossSpec("iid", 0.2), 70 + W))
 
 
+def test_random_shapes():
+    """Forty seeded random plans: tensor counts and sizes (tiny, ragged, exact multiples of a chunk, large), payload
+    sizes from 16 B to 64 KiB, 1 to 40 workers, both dtypes, every loss process."""
+    rng = np.random.default_rng(2024)
+    for case in range(40):
+        P = int(rng.choice([16, 48, 256, 1024, 1408, 2048, 4096, 8192, 65536]))
+        dtype = str(rng.choice(["f32", "bf16"]))
+        E = P // (4 if dtype == "f32" else 2)
+        numel = []
+        for _ in range(int(rng.integers(1, 13))):
+            kind = rng.integers(0, 4)
+            if kind == 0:
+                numel.append(int(rng.integers(1, 50)))
+            elif kind == 1:
+                numel.append(int(rng.integers(100, 5000)))
+            elif kind == 2:
+                numel.append(E * int(rng.integers(1, 6)))
+            else:
+                numel.append(int(rng.integers(5000, 200000)))
+        W = int(rng.integers(1, 41))
+        loss = [wl.LossSpec("none"), wl.LossSpec("iid", float(rng.uniform(0, 0.6))),
+                wl.LossSpec("ge", float(rng.uniform(0.01, 0.5)), float(rng.uniform(1.0, 30.0))),
+                wl.LossSpec("microburst", window_frac=float(rng.uniform(0, 1)), p_in=float(rng.uniform(0, 1)),
+                            p_out=float(rng.uniform(0, 0.2)))][int(rng.integers(0, 4))]
+        try:
+            H.full_round_parity(work(numel, dtype, P, W, loss, 1000 + case, bounds=(int(rng.integers(0, 500000)),)))
+        except AssertionError as e:
+            raise AssertionError("case %d: P=%d %s W=%d numel=%s loss=%s: %s" % (case, P, dtype, W, numel, loss, e))
+
+
 def test_thousands_of_workers_take_the_simple_reduce_kernel():
     """More workers than one chunk's slot entries fit in shared memory: the reduce falls back to its simple form, the
     fused extras say so instead of running, packetize goes through its worker groups."""
