@@ -165,14 +165,20 @@ def run_gpu(args):
         else:
             lossy_channel(rnd, ev)
         if ev: ev[2].record()
-        dblp.dblp_aggregate_book(plan, buf["hdr_ring"], plan.M, buf["arrival"], buf["n_arrived"], plan.M, rnd,
-                                 buf["recv_bitmap"], buf["slot_key"], buf["counters"])
+        if side is None:
+            dblp.dblp_aggregate_book(plan, buf["hdr_ring"], plan.M, buf["arrival"], buf["n_arrived"], plan.M, rnd,
+                                     buf["recv_bitmap"], buf["slot_key"], buf["counters"])
+        else:
+            dblp.dblp_aggregate_claim(plan, buf["hdr_ring"], plan.M, buf["arrival"], buf["n_arrived"], plan.M, rnd,
+                                      buf["slot_key"], buf["counters"])
         if ev: ev[3].record()
-        if side is not None:                           # the tolerance test needs the bitmap only: beside the reduce
+        if side is not None:                           # bitmap and tolerance test need the claims only: beside the reduce
             booked.record()
             with torch.cuda.stream(side):
                 side.wait_event(booked)
                 if ev: ev[8].record()
+                dblp.dblp_aggregate_bitmap(plan, buf["slot_key"], buf["n_arrived"], plan.M, buf["recv_bitmap"],
+                                           buf["counters"])
                 dblp.dblp_check_bound(plan, buf["recv_bitmap"], bound, buf["recv_cnt"], buf["missing_cnt"], buf["ok"],
                                       buf["all_ok"])
                 if ev: ev[5].record()
@@ -345,7 +351,7 @@ def run_gpu(args):
         "config": {"workload": work.name, "W": work.W, "payload_bytes": work.payload_bytes, "tensors": len(work.numel),
                    "elements_per_worker": work.N, "packets": plan.M, "loss": work.loss.kind,
                    "realised_loss": 1.0 - n_arrived / plan.M, "bound_ppm": bound, "reduce": "mean, fixed worker order",
-                   "streams": "one" if side is None else "apply_loss beside packetize and check_bound beside the reduce, on a high-priority side stream",
+                   "streams": "one" if side is None else "apply_loss beside packetize, bitmap + check_bound beside the reduce, on a high-priority side stream",
                    "l2": "inputs per step (%.0f MB) exceed the 126 MB L2; no flush" % (bytes_["total"] / 1e6),
                    "parallelism": "independent server shard per GPU" if world > 1 else "1 GPU"},
         "bytes_per_step": bytes_, "stage_ms": stage_ms,

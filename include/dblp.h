@@ -195,6 +195,16 @@ int dblp_apply_loss_static(const dblp_plan_t* plan, const dblp_loss_model_t* mod
  * The destination is the plan's (tensor base + chunk offset), never the slot's position.  agg_out: N fp32.
  *
  * dblp_aggregate runs both.  slot_key, recv_bitmap and counters are in/out round state (dblp_round_reset). */
+/* dblp_aggregate_book = dblp_aggregate_claim (examine the arrivals, claim cells, count) followed by
+ * dblp_aggregate_bitmap (rewrite recv_bitmap from slot_key and fold this call's arrival count into counters->n_arrived).
+ * The reduce needs only the claims, the tolerance test only the bitmap, so a caller with two streams can run the
+ * bitmap and dblp_check_bound beside dblp_aggregate_reduce.  Call dblp_aggregate_bitmap exactly once after each
+ * dblp_aggregate_claim, with the same n_arrived_dev and arrival_cap, before the round's next claim. */
+int dblp_aggregate_claim(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, uint64_t n_slots, const uint32_t* arrival,
+                         const uint64_t* n_arrived_dev, uint64_t arrival_cap, uint32_t round, uint64_t* slot_key,
+                         dblp_counters_t* counters, void* stream);
+int dblp_aggregate_bitmap(const dblp_plan_t* plan, const uint64_t* slot_key, const uint64_t* n_arrived_dev,
+                          uint64_t arrival_cap, uint32_t* recv_bitmap, dblp_counters_t* counters, void* stream);
 int dblp_aggregate_book(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, uint64_t n_slots, const uint32_t* arrival,
                         const uint64_t* n_arrived_dev, uint64_t arrival_cap, uint32_t round, uint32_t* recv_bitmap,
                         uint64_t* slot_key, dblp_counters_t* counters, void* stream);

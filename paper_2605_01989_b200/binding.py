@@ -53,7 +53,7 @@ EXPORTS = ("dblp_plan_create", "dblp_plan_destroy", "dblp_plan_query", "dblp_pla
            "dblp_apply_loss_resend", "dblp_missing_bits", "dblp_stop_workspace_bytes", "dblp_aggregate_book_stop",
            "dblp_round_until_stop",
            "dblp_aggregate_book",
-           "dblp_aggregate_reduce", "dblp_aggregate_reduce_ex", "dblp_aggregate_reduce_atomic", "dblp_norm_scratch_count", "dblp_aggregate", "dblp_round_reset", "dblp_check_bound", "dblp_bound_ok", "dblp_clr",
+           "dblp_aggregate_claim", "dblp_aggregate_bitmap", "dblp_aggregate_reduce", "dblp_aggregate_reduce_ex", "dblp_aggregate_reduce_atomic", "dblp_norm_scratch_count", "dblp_aggregate", "dblp_round_reset", "dblp_check_bound", "dblp_bound_ok", "dblp_clr",
            "dblp_select_bound", "dblp_round_host", "dblp_strerror", "dblp_last_error", "dblp_launch_count")
 
 
@@ -248,6 +248,18 @@ def dblp_aggregate_book(plan, hdr_ring, n_slots, arrival, n_arrived_dev, arrival
     _check(lib().dblp_aggregate_book(plan.handle, _ptr(hdr_ring), C.c_uint64(n_slots), _ptr(arrival),
                                      _ptr(n_arrived_dev), C.c_uint64(arrival_cap), C.c_uint32(round), _ptr(recv_bitmap),
                                      _ptr(slot_key), _ptr(counters), _stream(stream)), "dblp_aggregate_book")
+
+
+def dblp_aggregate_claim(plan, hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, slot_key, counters,
+                         stream=None):
+    _check(lib().dblp_aggregate_claim(plan.handle, _ptr(hdr_ring), C.c_uint64(n_slots), _ptr(arrival), _ptr(n_arrived_dev),
+                                      C.c_uint64(arrival_cap), C.c_uint32(round), _ptr(slot_key), _ptr(counters),
+                                      _stream(stream)), "dblp_aggregate_claim")
+
+
+def dblp_aggregate_bitmap(plan, slot_key, n_arrived_dev, arrival_cap, recv_bitmap, counters, stream=None):
+    _check(lib().dblp_aggregate_bitmap(plan.handle, _ptr(slot_key), _ptr(n_arrived_dev), C.c_uint64(arrival_cap),
+                                       _ptr(recv_bitmap), _ptr(counters), _stream(stream)), "dblp_aggregate_bitmap")
 
 
 def dblp_aggregate_reduce(plan, payload_ring, slot_key, agg_out, flags=DBLP_SUM, stream=None):

@@ -893,30 +893,46 @@ int configure_reduce(dblp_plan* p, uint32_t ch_override, uint32_t grid_override)
 
 using namespace dblp;
 
+extern "C" int dblp_aggregate_claim(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, uint64_t n_slots,
+                                    const uint32_t* arrival, const uint64_t* n_arrived_dev, uint64_t arrival_cap,
+                                    uint32_t round, uint64_t* slot_key, dblp_counters_t* counters, void* stream)
+{
+    DBLP_REQUIRE(plan && hdr_ring && arrival && n_arrived_dev && slot_key && counters, DBLP_EINVAL,
+                 "aggregate_claim: null argument");
+    DBLP_REQUIRE(aligned16(hdr_ring), DBLP_EALIGN, "aggregate_claim: header ring must be 16-byte aligned");
+    DBLP_REQUIRE(n_slots < 0xFFFFFFFFull, DBLP_ECAPACITY, "aggregate_claim: ring has too many slots");
+    DBLP_REQUIRE(arrival_cap < (1ull << 32), DBLP_ECAPACITY, "aggregate_claim: arrival list too long");
+    if (arrival_cap == 0) return DBLP_OK;
+    const unsigned grid = (unsigned)((arrival_cap + kBookThreads - 1) / kBookThreads);
+    k_book<<<grid, kBookThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, reinterpret_cast<unsigned long long*>(slot_key), counters,
+        plan->d_numel, plan->d_chunkbase, plan->T, plan->W, plan->C, plan->E, plan->es, plan->hdr_stride);
+    DBLP_LAUNCHED();
+    return DBLP_OK;
+}
+
+extern "C" int dblp_aggregate_bitmap(const dblp_plan_t* plan, const uint64_t* slot_key, const uint64_t* n_arrived_dev,
+                                     uint64_t arrival_cap, uint32_t* recv_bitmap, dblp_counters_t* counters, void* stream)
+{
+    DBLP_REQUIRE(plan && slot_key && n_arrived_dev && recv_bitmap && counters, DBLP_EINVAL, "aggregate_bitmap: null argument");
+    const uint64_t cells = plan->row_words * 32 * plan->W;
+    k_bitmap<<<(unsigned)((cells + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        reinterpret_cast<const unsigned long long*>(slot_key), recv_bitmap, plan->W, plan->C, plan->row_words, n_arrived_dev,
+        arrival_cap, counters);
+    DBLP_LAUNCHED();
+    return DBLP_OK;
+}
+
 extern "C" int dblp_aggregate_book(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, uint64_t n_slots,
                                    const uint32_t* arrival, const uint64_t* n_arrived_dev, uint64_t arrival_cap,
                                    uint32_t round, uint32_t* recv_bitmap, uint64_t* slot_key, dblp_counters_t* counters,
                                    void* stream)
 {
-    DBLP_REQUIRE(plan && hdr_ring && arrival && n_arrived_dev && recv_bitmap && slot_key && counters, DBLP_EINVAL,
-                 "aggregate_book: null argument");
-    DBLP_REQUIRE(aligned16(hdr_ring), DBLP_EALIGN, "aggregate_book: header ring must be 16-byte aligned");
-    DBLP_REQUIRE(n_slots < 0xFFFFFFFFull, DBLP_ECAPACITY, "aggregate_book: ring has too many slots");
-    DBLP_REQUIRE(arrival_cap < (1ull << 32), DBLP_ECAPACITY, "aggregate_book: arrival list too long");
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (arrival_cap > 0) {
-        const unsigned grid = (unsigned)((arrival_cap + kBookThreads - 1) / kBookThreads);
-        k_book<<<grid, kBookThreads, 0, s>>>(hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round,
-                                             reinterpret_cast<unsigned long long*>(slot_key), counters, plan->d_numel,
-                                             plan->d_chunkbase, plan->T, plan->W, plan->C, plan->E, plan->es, plan->hdr_stride);
-        DBLP_LAUNCHED();
-    }
-    const uint64_t cells = plan->row_words * 32 * plan->W;
-    k_bitmap<<<(unsigned)((cells + 255) / 256), 256, 0, s>>>(reinterpret_cast<const unsigned long long*>(slot_key),
-                                                           recv_bitmap, plan->W, plan->C, plan->row_words,
-                                                           n_arrived_dev, arrival_cap, counters);
-    DBLP_LAUNCHED();
-    return DBLP_OK;
+    DBLP_REQUIRE(recv_bitmap, DBLP_EINVAL, "aggregate_book: null argument");
+    const int rc = dblp_aggregate_claim(plan, hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, slot_key,
+                                        counters, stream);
+    if (rc != DBLP_OK) return rc;
+    return dblp_aggregate_bitmap(plan, slot_key, n_arrived_dev, arrival_cap, recv_bitmap, counters, stream);
 }
 
 extern "C" int dblp_stop_workspace_bytes(const dblp_plan_t* plan, uint64_t arrival_cap, size_t* bytes)

@@ -337,6 +337,27 @@ def test_argument_errors_are_reported_not_faulted():
     g.close()
 
 
+def test_claim_then_bitmap_equals_book():
+    w = work(RAGGED, "f32", 1408, 4, wl.LossSpec("iid", 0.2), 61)
+    op = orc.Plan(w.numel, 4, 1408, 4)
+    gm, om = H.models_for(w, op.C)
+    g = H.GpuRound(w)
+    b = g.buf
+    g.packetize(wl.make_grads(w, H.DEV), w.round)
+    o_hdr = op.headers(w.round)
+    st = op.new_state()
+    for attempt in range(2):                                   # the second call sees cells already claimed
+        g.apply_loss(gm, w.seed, w.round, attempt)
+        dblp.dblp_aggregate_claim(g.plan, b["hdr_ring"], op.M, b["arrival"], b["n_arrived"], op.M, w.round, b["slot_key"],
+                                  b["counters"])
+        dblp.dblp_aggregate_bitmap(g.plan, b["slot_key"], b["n_arrived"], op.M, b["recv_bitmap"], b["counters"])
+        o_del, _ = op.loss_mask(om, w.seed, w.round, attempt)
+        o_arr, o_n = op.arrival(o_del, w.seed, w.round, attempt)
+        st = op.book(o_hdr, o_arr, o_n, w.round, st)
+        H.compare_state(g, st, op)
+    g.close()
+
+
 def test_library_counts_its_launches():
     w = work(ALIGNED, "f32", 1024, 2, wl.LossSpec("ge", 0.1, 5.0), 1)
     g = H.GpuRound(w)
