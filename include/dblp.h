@@ -115,7 +115,8 @@ int dblp_plan_set_wire_format(dblp_plan_t* plan, int format);
  * DBLP_ECAPACITY if the tile's slot entries do not fit in shared memory.  Not to be called while work that uses the
  * plan is being enqueued from another thread. */
 int dblp_plan_tune_reduce(dblp_plan_t* plan, uint32_t chunks_per_tile, uint32_t grid_blocks);
-/* Bytes of scratch that dblp_apply_loss needs (the other calls need none). */
+/* Bytes of scratch that dblp_apply_loss / dblp_apply_loss_resend need.  dblp_aggregate_book_stop has its own query
+ * (dblp_stop_workspace_bytes); the remaining calls need none. */
 int dblp_workspace_bytes(const dblp_plan_t* plan, size_t* bytes);
 
 /* HOST helper: rates -> thresholds floor(prob * 2^32).  IID uses mean_loss.  GE is the simple Gilbert chain
