@@ -392,7 +392,7 @@ def run_gpu(args):
         "aggregate_path": {"what": "bookkeeping + masked reduce + bound check only", "GBps": agg_gbs, "ms": agg_ms,
                            "pct_of_nominal_8TBs": 100.0 * agg_gbs / NOMINAL_HBM_GBS,
                            "pct_of_%s_peak" % peak_kind: 100.0 * agg_gbs / peak},
-        "roofline": {"kernel": "k_reduce_tiled", "bound": "hbm", "achieved": red_gbs, "peak": peak, "peak_kind": peak_kind,
+        "roofline": {"kernel": "k_reduce_rows" if work.W <= 4 and work.payload_bytes >= 2048 else "k_reduce_tiled", "bound": "hbm", "achieved": red_gbs, "peak": peak, "peak_kind": peak_kind,
                      "unit": "GB/s", "frac": red_gbs / peak, "traffic": TRAFFIC.get(work.name),
                      "algorithmic_bytes_per_launch": bytes_["reduce"], "ms_per_launch": stage_ms["reduce"]},
         "clocks": clocks, "gpu_launches": launches, "e2e": e2e, "cpu_baseline": cpu, "round_loop": round_loop, "reduce_extras": extras,
