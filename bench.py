@@ -273,7 +273,9 @@ def run_gpu(args):
 
     # end to end from host memory: pinned gradients in, aggregate + counts out, every step
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and work.W * work.N * work.elem_size > (16 << 30):
+        e2e = {"skipped": "host copies of %.0f GB of gradients: run with a smaller workload" % (work.W * work.N * work.elem_size / 1e9)}
+    elif not args.no_e2e:
         grads_host = [g.cpu().pin_memory() for g in grads]
         grads_dev = torch.empty(work.W * work.N, dtype=plan.torch_dtype, device=dev)
         agg_host = torch.empty(work.N, dtype=torch.float32).pin_memory()
