@@ -2,18 +2,24 @@
  * dblp.h -- C ABI of libdblp: the receive-side data path of the Dynamic Bounded-Loss Protocol (DBLP)
  * for W simulated workers whose gradients are resident on one CUDA device (sm_100a).
  *
- * One communication round is four calls on one stream:
+ * One communication round is four steps:
  *
  *   dblp_packetize   gradients            -> header ring + payload ring      (Algorithm 1, first step)
  *   dblp_apply_loss  seeded loss process  -> delivered bitmap + arrival list (Sections II-C, V-B; property 1)
  *   dblp_aggregate   arrival list + rings -> received bitmap + aggregate     (Algorithm 2; Algorithm 3 "mean")
  *   dblp_check_bound received bitmap      -> per-worker loss counts, stop / continue decision (Section III-B)
  *
+ * Each is a call of its own on the caller's stream.  dblp_round_device runs all four as one call and overlaps what is
+ * independent: apply_loss (ALU-bound) beside packetize (HBM-bound), and the bitmap + tolerance test beside the masked
+ * reduce, on a high-priority stream that the plan owns; dblp_round_host does the same from host buffers with the
+ * copies overlapped.  Results are identical either way.
+ *
  * Conventions
  *   - Every function returns DBLP_OK (0) or a negative dblp_status_t; nothing throws, aborts or traps.
  *     dblp_last_error() gives the text of the calling thread's most recent failure.
  *   - Unless an argument is marked HOST it is a DEVICE pointer owned by the caller, on the device that was
- *     current when the plan was created.  The library allocates device memory only in dblp_plan_create.
+ *     current when the plan was created.  The library allocates device memory, streams and events only in
+ *     dblp_plan_create.
  *   - Per-round calls only enqueue work on the given stream (a cudaStream_t passed as void*; NULL = the
  *     legacy default stream) and do not synchronise.  Counts that a later step needs stay on the device.
  *   - Anomalies found on the device (bad slot index, header that contradicts the plan, wrong round, repeated
@@ -78,7 +84,9 @@ typedef struct {
     uint64_t t_drop_in, t_drop_out;
 } dblp_loss_model_t;
 
-/* Receiver statistics of a round (device memory; all fields accumulate until dblp_round_reset). */
+/* Receiver statistics of a round (device memory; all fields accumulate until dblp_round_reset).  n_accepted and n_dup
+ * are settled by the bitmap step of the bookkeeping (dblp_aggregate_bitmap): between a dblp_aggregate_claim and its
+ * dblp_aggregate_bitmap every valid packet of the call is still counted under n_dup. */
 typedef struct {
     uint64_t n_arrived;  /* arrival-list entries examined */
     uint64_t n_accepted; /* packets whose bit was newly set */
@@ -110,6 +118,15 @@ int dblp_plan_query(const dblp_plan_t* plan, uint64_t* C, uint64_t* N, uint64_t*
  * payload_ring to every call.  Set before the first round; results do not depend on it. */
 enum { DBLP_WIRE_RINGS = 0, DBLP_WIRE_DATAGRAMS = 1 };
 int dblp_plan_set_wire_format(dblp_plan_t* plan, int format);
+/* A server split over several devices (Section IV-D's server, sharded by offset range): each device owns a contiguous
+ * run of the tensors with a plan of its own, whose packets are the chunks seq_offset .. seq_offset + C - 1 of worker
+ * streams that are stream_chunks long in all.  After this call the loss process draws each packet's fate by its number
+ * in the whole stream (and runs the burst chain and places the microburst window along the whole stream), so that the
+ * shards' delivered bitmaps, side by side, are exactly the delivered bitmap of the unsplit round.  Headers, sequence
+ * numbers and the arrival permutation stay local to the shard.  dblp_workspace_bytes grows by one stream-wide bitmap.
+ * dblp_apply_loss_resend with a send set and DBLP_LOSS_GE is refused on such a plan (DBLP_EINVAL): the chain would need
+ * the send set of the whole stream.  Call before the first round. */
+int dblp_plan_set_shard(dblp_plan_t* plan, uint64_t stream_chunks, uint64_t seq_offset);
 /* Expert knob: pins the launch shape of the masked reduce (dblp_aggregate_reduce) -- chunks summed per tile and
  * number of persistent blocks; 0 = choose automatically (what dblp_plan_create does).  Results do not depend on it.
  * DBLP_ECAPACITY if the tile's slot entries do not fit in shared memory.  Not to be called while work that uses the
@@ -121,7 +138,8 @@ int dblp_workspace_bytes(const dblp_plan_t* plan, size_t* bytes);
 
 /* HOST helper: rates -> thresholds floor(prob * 2^32).  IID uses mean_loss.  GE is the simple Gilbert chain
  * (every packet sent in Bad is lost): P(Bad->Good) = 1 / mean_burst_len, P(Good->Bad) chosen so the stationary loss
- * is mean_loss, start state drawn from the stationary law.  MICROBURST: window_len = ceil(window_frac * C). */
+ * is mean_loss, start state drawn from the stationary law; DBLP_EINVAL if that P(Good->Bad) would exceed 1 (the mean
+ * loss cannot be reached with bursts that short).  MICROBURST: window_len = ceil(window_frac * C). */
 int dblp_loss_model_from_rates(int kind, double mean_loss, double mean_burst_len, double window_frac, double p_in,
                                double p_out, uint64_t C, dblp_loss_model_t* out);
 
@@ -196,8 +214,10 @@ int dblp_apply_loss_static(const dblp_plan_t* plan, const dblp_loss_model_t* mod
  * The destination is the plan's (tensor base + chunk offset), never the slot's position.  agg_out: N fp32.
  *
  * dblp_aggregate runs both.  slot_key, recv_bitmap and counters are in/out round state (dblp_round_reset). */
-/* dblp_aggregate_book = dblp_aggregate_claim (examine the arrivals, claim cells, count) followed by
- * dblp_aggregate_bitmap (rewrite recv_bitmap from slot_key and fold this call's arrival count into counters->n_arrived).
+/* dblp_aggregate_book = dblp_aggregate_claim (examine the arrivals, claim cells, count stale and invalid ones) followed
+ * by dblp_aggregate_bitmap (rewrite recv_bitmap from slot_key; the bits that are new are the packets accepted by this
+ * call, the other valid ones were repeats; fold this call's arrival count into counters->n_arrived).  recv_bitmap must
+ * be the round's bitmap as the previous bookkeeping call (or dblp_round_reset) left it.
  * The reduce needs only the claims, the tolerance test only the bitmap, so a caller with two streams can run the
  * bitmap and dblp_check_bound beside dblp_aggregate_reduce.  Call dblp_aggregate_bitmap exactly once after each
  * dblp_aggregate_claim, with the same n_arrived_dev and arrival_cap, before the round's next claim. */
@@ -282,13 +302,10 @@ int dblp_clr(double norm_prev, double norm_curr, double eta);
 uint32_t dblp_select_bound(double norm_prev, double norm_curr, double eta, uint32_t p_low_ppm, uint32_t p_high_ppm,
                            int at_epoch_start, int first_iteration, uint32_t current_ppm);
 
-/* ---- one whole round from HOST buffers --------------------------------------------------------------------------
- * Copies each worker's gradient from host memory (pinned memory recommended) into dev->grads, runs
- * round_reset, packetize, apply_loss, aggregate and check_bound, copies the aggregate, the counters and the bound
- * outputs back to the host pointers and waits for the stream.  Every member of dblp_device_buffers_t is a device
- * buffer the caller allocated with the sizes given; nothing is allocated here.  Host outputs may be NULL to skip. */
+/* ---- whole rounds ---------------------------------------------------------------------------------------------------
+ * The device buffers of a round, all allocated by the caller with the sizes given. */
 typedef struct {
-    void* grads;               /* W * N elements of the plan's dtype, worker-major */
+    void* grads;               /* W * N elements of the plan's dtype, worker-major; dblp_round_host only */
     dblp_hdr_t* hdr_ring;      /* M headers */
     void* payload_ring;        /* M * payload_bytes */
     uint32_t* delivered_bits;  /* W * row_words */
@@ -302,11 +319,49 @@ typedef struct {
     uint32_t* missing_cnt;     /* W * B */
     uint8_t* ok;               /* W * B */
     uint32_t* all_ok;          /* 1 */
-    void* ws;                  /* max(dblp_workspace_bytes, dblp_stop_workspace_bytes(M)) when dblp_round_until_stop uses it */
+    void* ws;                  /* dblp_workspace_bytes (max with dblp_stop_workspace_bytes(M) for dblp_round_until_stop) */
     size_t ws_bytes;
     uint32_t* sent_bits;       /* W * row_words; used by dblp_round_until_stop only */
 } dblp_device_buffers_t;
 
+/* Optional stage marks: CUDA events (cudaEvent_t passed as void*, created by the caller) that a whole-round call
+ * records where a stage begins or ends, on the stream that runs the stage, so that a caller can time the stages of the
+ * overlapped schedule.  NULL members are skipped; a NULL struct pointer means no marks. */
+typedef struct {
+    void* begin;          /* caller's stream, before anything */
+    void* packetize_end;  /* caller's stream */
+    void* loss_begin;     /* side stream: round_reset + apply_loss */
+    void* loss_end;
+    void* receive_begin;  /* caller's stream, once packetize and apply_loss have both finished */
+    void* claim_end;      /* caller's stream: arrivals examined, cells claimed */
+    void* reduce_end;     /* caller's stream */
+    void* bound_begin;    /* side stream: bitmap + check_bound */
+    void* bound_end;
+    void* end;            /* caller's stream, after the side stream has been joined */
+} dblp_round_marks_t;
+
+/* dblp_round_device = one round of the server on gradients resident in device memory (Algorithm 3: receive from
+ * every worker, then the mean; Algorithm 2 inside; Section III-B for the tolerance test):
+ *   dblp_round_send     round_reset and apply_loss (attempt 0) on the plan's side stream beside dblp_packetize on the
+ *                       caller's stream; returns with the caller's stream waiting for both.
+ *   dblp_round_receive  dblp_aggregate_claim, then dblp_aggregate_bitmap + dblp_check_bound (one tolerance for all) on
+ *                       the side stream beside dblp_aggregate_reduce; the caller's stream waits for both at the end.
+ * grads: HOST array of W device pointers as for dblp_packetize.  flags: DBLP_SUM or DBLP_MEAN.  Packets occupy ring slots
+ * 0 .. M-1.  Nothing is allocated and the host is not blocked.  The side stream and its events belong to the plan, so a
+ * plan serves one whole-round call at a time (calls on one stream, or ordered by the caller). */
+int dblp_round_send(const dblp_plan_t* plan, const void* const* grads, const dblp_loss_model_t* model, uint64_t seed,
+                    uint32_t round, const dblp_device_buffers_t* dev, const dblp_round_marks_t* marks, void* stream);
+int dblp_round_receive(const dblp_plan_t* plan, uint32_t round, uint32_t bound_ppm, uint32_t flags,
+                       const dblp_device_buffers_t* dev, const dblp_round_marks_t* marks, void* stream);
+int dblp_round_device(const dblp_plan_t* plan, const void* const* grads, const dblp_loss_model_t* model, uint64_t seed,
+                      uint32_t round, uint32_t bound_ppm, uint32_t flags, const dblp_device_buffers_t* dev,
+                      const dblp_round_marks_t* marks, void* stream);
+
+/* dblp_round_host = the same round from HOST gradients (grads_host: HOST array of W host pointers, pinned memory
+ * recommended): worker w's gradient is copied into dev->grads on the plan's copy stream while worker w - 1 is being
+ * packetized, the loss process runs beside both, then dblp_round_receive; the aggregate, the counters and the bound
+ * outputs are copied back to the host pointers (NULL to skip) and the call waits for the stream.  Nothing is
+ * allocated. */
 int dblp_round_host(const dblp_plan_t* plan, const void* const* grads_host, const dblp_loss_model_t* model,
                     uint64_t seed, uint32_t round, uint32_t bound_ppm, uint32_t flags,
                     const dblp_device_buffers_t* dev, float* agg_host, dblp_counters_t* counters_host,

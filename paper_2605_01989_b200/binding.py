@@ -39,6 +39,27 @@ class dblp_device_buffers_t(C.Structure):
                                                                                    ("sent_bits", C.c_void_p)]
 
 
+MARK_FIELDS = ("begin", "packetize_end", "loss_begin", "loss_end", "receive_begin", "claim_end", "reduce_end",
+               "bound_begin", "bound_end", "end")
+
+
+class dblp_round_marks_t(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in MARK_FIELDS]
+
+
+class RoundMarks:
+    """Timing events for the stages of a whole-round call (torch events; the library records them)."""
+
+    def __init__(self):
+        self.events = {n: torch.cuda.Event(enable_timing=True) for n in MARK_FIELDS}
+        for e in self.events.values():
+            e.record()                      # torch creates the CUDA event on first use; the library needs the handle
+        self.struct = dblp_round_marks_t(**{n: e.cuda_event for n, e in self.events.items()})
+
+    def ms(self, first, last):
+        return self.events[first].elapsed_time(self.events[last])
+
+
 class DblpError(RuntimeError):
     def __init__(self, status, what):
         super().__init__("%s: %s (%d): %s" % (what, lib().dblp_strerror(status).decode(), status,
@@ -48,13 +69,15 @@ class DblpError(RuntimeError):
 
 _lib = None
 EXPORTS = ("dblp_plan_create", "dblp_plan_destroy", "dblp_plan_query", "dblp_plan_tune_reduce", "dblp_plan_set_wire_format",
+           "dblp_plan_set_shard",
            "dblp_workspace_bytes",
            "dblp_loss_model_from_rates", "dblp_packetize", "dblp_apply_loss", "dblp_apply_loss_static",
            "dblp_apply_loss_resend", "dblp_missing_bits", "dblp_stop_workspace_bytes", "dblp_aggregate_book_stop",
            "dblp_round_until_stop",
            "dblp_aggregate_book",
            "dblp_aggregate_claim", "dblp_aggregate_bitmap", "dblp_aggregate_reduce", "dblp_aggregate_reduce_ex", "dblp_aggregate_reduce_atomic", "dblp_norm_scratch_count", "dblp_aggregate", "dblp_round_reset", "dblp_check_bound", "dblp_bound_ok", "dblp_clr",
-           "dblp_select_bound", "dblp_round_host", "dblp_strerror", "dblp_last_error", "dblp_launch_count")
+           "dblp_select_bound", "dblp_round_send", "dblp_round_receive", "dblp_round_device", "dblp_round_host",
+           "dblp_strerror", "dblp_last_error", "dblp_launch_count")
 
 
 def lib():
@@ -140,6 +163,13 @@ class Plan:
         """True: one ring of (32 + P)-byte datagrams (pass it as both hdr_ring and payload_ring); False: two rings."""
         _check(lib().dblp_plan_set_wire_format(self.handle, C.c_int(1 if datagrams else 0)), "dblp_plan_set_wire_format")
         self.datagrams = bool(datagrams)
+
+    def set_shard(self, stream_chunks, seq_offset):
+        """This plan is the chunks seq_offset .. seq_offset + C - 1 of worker streams of stream_chunks chunks."""
+        _check(lib().dblp_plan_set_shard(self.handle, C.c_uint64(stream_chunks), C.c_uint64(seq_offset)), "dblp_plan_set_shard")
+        ws = C.c_size_t()
+        _check(lib().dblp_workspace_bytes(self.handle, C.byref(ws)), "dblp_workspace_bytes")
+        self.workspace_bytes = int(ws.value)
 
     def tune_reduce(self, chunks_per_tile=0, grid_blocks=0):
         _check(lib().dblp_plan_tune_reduce(self.handle, C.c_uint32(chunks_per_tile), C.c_uint32(grid_blocks)),
@@ -316,6 +346,34 @@ def dblp_clr(norm_prev, norm_curr, eta=0.5):
 def dblp_select_bound(norm_prev, norm_curr, eta, p_low_ppm, p_high_ppm, at_epoch_start, first_iteration, current_ppm):
     return int(lib().dblp_select_bound(norm_prev, norm_curr, eta, p_low_ppm, p_high_ppm, int(at_epoch_start),
                                        int(first_iteration), current_ppm))
+
+
+def _marks(marks):
+    return C.byref(marks.struct) if marks is not None else None
+
+
+def _grad_ptrs(plan, grads):
+    return (C.c_void_p * plan.W)(*[g.data_ptr() for g in grads])
+
+
+def dblp_round_send(plan, grads, model, seed, round, dev, marks=None, stream=None):
+    b = _device_buffers(dev)
+    _check(lib().dblp_round_send(plan.handle, _grad_ptrs(plan, grads), C.byref(model), C.c_uint64(seed), C.c_uint32(round),
+                                 C.byref(b), _marks(marks), _stream(stream)), "dblp_round_send")
+
+
+def dblp_round_receive(plan, round, bound_ppm, flags, dev, marks=None, stream=None):
+    b = _device_buffers(dev)
+    _check(lib().dblp_round_receive(plan.handle, C.c_uint32(round), C.c_uint32(bound_ppm), C.c_uint32(flags), C.byref(b),
+                                    _marks(marks), _stream(stream)), "dblp_round_receive")
+
+
+def dblp_round_device(plan, grads, model, seed, round, bound_ppm, flags, dev, marks=None, stream=None):
+    """One whole round on device-resident gradients with the library's two-stream schedule."""
+    b = _device_buffers(dev)
+    _check(lib().dblp_round_device(plan.handle, _grad_ptrs(plan, grads), C.byref(model), C.c_uint64(seed),
+                                   C.c_uint32(round), C.c_uint32(bound_ppm), C.c_uint32(flags), C.byref(b),
+                                   _marks(marks), _stream(stream)), "dblp_round_device")
 
 
 def dblp_round_host(plan, grads_host, model, seed, round, bound_ppm, flags, dev, grads_dev, agg_host=None,

@@ -26,71 +26,137 @@ constexpr int kReduceThreads = 256;
 constexpr int kWorkerBatch = 8;
 
 // ------------------------------------------------------------------------------------------------ bookkeeping
+// Algorithm 2's integrity check, shared by both claim kernels: the slot must lie inside the ring and the header must
+// agree with the plan (worker < W, tensor < T, offset on a chunk boundary inside the tensor, length and sequence
+// number those of that chunk).  tensor_tab[t] = (numel low, numel high, first sequence number, 0): one 16-byte load
+// behind the header instead of two dependent ones.
+struct HeaderView {
+    bool valid;          // passes the integrity check
+    uint32_t worker, seq, round;
+};
+
+__device__ __forceinline__ HeaderView validate_header(const dblp_hdr_t* __restrict__ hdr_ring, uint32_t hdr_stride,
+                                                      uint32_t slot, uint64_t n_slots,
+                                                      const uint4* __restrict__ tensor_tab, uint32_t T, uint32_t W,
+                                                      uint32_t E, uint32_t es)
+{
+    HeaderView h{false, 0u, 0u, 0u};
+    if (slot >= n_slots) return h;
+    const uint4* hp = reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(hdr_ring) + (uint64_t)slot * hdr_stride);
+    const uint4 h0 = __ldg(hp);       // seq, round, len_bytes, tensor_id
+    const uint4 h1 = __ldg(hp + 1);   // offset low, offset high, worker, reserved
+    h.worker = h1.z; h.seq = h0.x; h.round = h0.y;
+    if (h1.z >= W || h0.w >= T) return h;
+    const uint4 tt = __ldg(&tensor_tab[h0.w]);
+    const uint64_t nt = (uint64_t)tt.x | ((uint64_t)tt.y << 32);
+    const uint64_t off = (uint64_t)h1.x | ((uint64_t)h1.y << 32);
+    if (off >= nt) return h;
+    uint64_t q;
+    bool on_boundary;
+    if (h1.y == 0) {                  // offsets below 2^32 (all but the largest tensors): 32-bit division
+        const uint32_t q32 = h1.x / E;
+        on_boundary = q32 * E == h1.x;
+        q = q32;
+    } else {
+        q = off / E;
+        on_boundary = q * E == off;
+    }
+    const uint64_t len = min((uint64_t)E, nt - off);
+    h.valid = on_boundary && (h0.z == len * es) && (h0.x == tt.z + q);
+    return h;
+}
+
+// Block-wide counts of three per-thread flags: warp ballots, one shared-memory atomic per warp and non-zero count.
+// Every thread of the block must call it.
+__device__ __forceinline__ void block_count3(bool a, bool b, bool c, uint32_t* s_cnt)
+{
+    if (threadIdx.x < 3) s_cnt[threadIdx.x] = 0;
+    __syncthreads();
+    const uint32_t na = __popc(__ballot_sync(0xFFFFFFFFu, a));
+    const uint32_t nb = __popc(__ballot_sync(0xFFFFFFFFu, b));
+    const uint32_t nc = __popc(__ballot_sync(0xFFFFFFFFu, c));
+    if ((threadIdx.x & 31) == 0) {
+        if (na) atomicAdd(&s_cnt[0], na);
+        if (nb) atomicAdd(&s_cnt[1], nb);
+        if (nc) atomicAdd(&s_cnt[2], nc);
+    }
+    __syncthreads();
+}
+
+// One thread per arrival entry.  The claim is a 64-bit atomic minimum that nobody waits for (no return value): who
+// won a cell is settled by the minimum itself, and how many cells were newly won is counted afterwards by k_bitmap from
+// the bitmap words it rewrites.  Here every valid packet of this round is provisionally counted as a repeat
+// (n_dup); k_bitmap moves the newly set bits from n_dup to n_accepted.
 __global__ void __launch_bounds__(kBookThreads)
 k_book(const dblp_hdr_t* __restrict__ hdr_ring, uint64_t n_slots, const uint32_t* __restrict__ arrival,
        const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap, uint32_t round,
        unsigned long long* __restrict__ slot_key, dblp_counters_t* counters,
-       const uint64_t* __restrict__ numel, const uint32_t* __restrict__ chunkbase,
-       uint32_t T, uint32_t W, uint64_t C, uint32_t E, uint32_t es, uint32_t hdr_stride)
+       const uint4* __restrict__ tensor_tab, uint32_t T, uint32_t W, uint64_t C, uint32_t E, uint32_t es,
+       uint32_t hdr_stride)
 {
+    __shared__ uint32_t s_cnt[3];
     const uint64_t n = min(*n_arrived_dev, arrival_cap);
     const uint64_t a = (uint64_t)blockIdx.x * kBookThreads + threadIdx.x;
     if ((uint64_t)blockIdx.x * kBookThreads >= n) return;          // whole block past the end
     const uint64_t first_number = counters->n_arrived;             // arrival numbers continue across calls of a round
-    int accepted = 0, dup = 0, stale = 0, invalid = 0;
+    bool current = false, stale = false, invalid = false;
     if (a < n) {
         const uint32_t slot = __ldg(&arrival[a]);
-        bool valid = false;
-        uint4 h0 = make_uint4(0, 0, 0, 0), h1 = h0;
-        if (slot < n_slots) {
-            const uint4* hp = reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(hdr_ring) + (uint64_t)slot * hdr_stride);
-            h0 = __ldg(hp);       // seq, round, len_bytes, tensor_id
-            h1 = __ldg(hp + 1);   // offset lo, offset hi, worker, reserved
-            const uint64_t off = (uint64_t)h1.x | ((uint64_t)h1.y << 32);
-            if (h1.z < W && h0.w < T) {
-                const uint64_t nt = __ldg(&numel[h0.w]);
-                if (off < nt && off % E == 0) {
-                    const uint64_t len = min((uint64_t)E, nt - off);
-                    valid = (h0.z == len * es) && (h0.x == __ldg(&chunkbase[h0.w]) + off / E);
-                }
-            }
-        }
-        if (!valid) invalid = 1;
-        else if (h0.y != round) stale = 1;
+        const HeaderView h = validate_header(hdr_ring, hdr_stride, slot, n_slots, tensor_tab, T, W, E, es);
+        if (!h.valid) invalid = true;
+        else if (h.round != round) stale = true;
         else {
-            const unsigned long long key = ((first_number + a) << 32) | slot;
-            const unsigned long long old = atomicMin(&slot_key[(uint64_t)h1.z * C + h0.x], key);
-            if (old == kEmpty64) accepted = 1; else dup = 1;
+            current = true;
+            atomicMin(&slot_key[(uint64_t)h.worker * C + h.seq], ((first_number + a) << 32) | slot);
         }
     }
-    const int n_acc = __syncthreads_count(accepted), n_dup = __syncthreads_count(dup);
-    const int n_stale = __syncthreads_count(stale), n_inv = __syncthreads_count(invalid);
+    block_count3(current, stale, invalid, s_cnt);
     if (threadIdx.x == 0) {
-        if (n_acc) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_accepted), (unsigned long long)n_acc);
-        if (n_dup) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_dup), (unsigned long long)n_dup);
-        if (n_stale) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_stale), (unsigned long long)n_stale);
-        if (n_inv) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_invalid), (unsigned long long)n_inv);
+        if (s_cnt[0]) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_dup), (unsigned long long)s_cnt[0]);
+        if (s_cnt[1]) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_stale), (unsigned long long)s_cnt[1]);
+        if (s_cnt[2]) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_invalid), (unsigned long long)s_cnt[2]);
     }
 }
 
+// Rewrites the received bitmap from the claim table (warp ballot -> one word per warp) and folds this call's arrival
+// count into the counters (after every k_book thread has read the old value).  With count_new set, the bits that are
+// new in each word are the cells k_book's claims have just won: they move from n_dup to n_accepted.
 __global__ void __launch_bounds__(256)
 k_bitmap(const unsigned long long* __restrict__ slot_key, uint32_t* __restrict__ recv_bitmap, uint32_t W, uint64_t C,
-         uint64_t row_words, const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap, dblp_counters_t* counters)
+         uint64_t row_words, const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap, dblp_counters_t* counters,
+         int count_new)
 {
+    __shared__ uint32_t s_new;
     const uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;   // (row, word, lane)
     const uint64_t row_bits = row_words * 32;
+    if (threadIdx.x == 0) s_new = 0;
     if (i == 0) {
         const uint64_t total = counters->n_arrived + min(*n_arrived_dev, arrival_cap);
         counters->n_arrived = total;
         if (total > 0xFFFFFFFFull) counters->status |= 1u;
     }
-    if (i >= row_bits * W) return;            // row_bits is a multiple of 32: whole warps leave together
-    const uint32_t w = (uint32_t)(i / row_bits);
-    const uint64_t c = i - (uint64_t)w * row_bits;
-    bool got = false;
-    if (c < C) got = reinterpret_cast<const uint2*>(slot_key)[(uint64_t)w * C + c].x != kEmpty32;
-    const uint32_t word = __ballot_sync(0xFFFFFFFFu, got);
-    if ((threadIdx.x & 31) == 0) recv_bitmap[(uint64_t)w * row_words + (c >> 5)] = word;
+    __syncthreads();
+    if (i < row_bits * W) {                   // row_bits is a multiple of 32: whole warps are in or out together
+        const uint32_t w = (uint32_t)(i / row_bits);
+        const uint64_t c = i - (uint64_t)w * row_bits;
+        bool got = false;
+        if (c < C) got = reinterpret_cast<const uint2*>(slot_key)[(uint64_t)w * C + c].x != kEmpty32;
+        const uint32_t word = __ballot_sync(0xFFFFFFFFu, got);
+        if ((threadIdx.x & 31) == 0) {
+            uint32_t* dst = &recv_bitmap[(uint64_t)w * row_words + (c >> 5)];
+            if (count_new) {
+                const uint32_t fresh = __popc(word & ~*dst);
+                if (fresh) atomicAdd(&s_new, fresh);
+            }
+            *dst = word;
+        }
+    }
+    if (!count_new) return;
+    __syncthreads();
+    if (threadIdx.x == 0 && s_new) {
+        atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_accepted), (unsigned long long)s_new);
+        atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_dup), 0ull - (unsigned long long)s_new);
+    }
 }
 
 // ------------------------------------------------------------------------------------------------ early stop
@@ -126,44 +192,31 @@ __global__ void __launch_bounds__(kBookThreads)
 k_book_claim(const dblp_hdr_t* __restrict__ hdr_ring, uint64_t n_slots, const uint32_t* __restrict__ arrival,
              const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap, uint32_t round,
              unsigned long long* __restrict__ slot_key, dblp_counters_t* counters, uint32_t* __restrict__ cell_of,
-             const uint64_t* __restrict__ numel, const uint32_t* __restrict__ chunkbase,
-             uint32_t T, uint32_t W, uint64_t C, uint32_t E, uint32_t es, uint32_t hdr_stride)
+             const uint4* __restrict__ tensor_tab, uint32_t T, uint32_t W, uint64_t C, uint32_t E, uint32_t es,
+             uint32_t hdr_stride)
 {
+    __shared__ uint32_t s_cnt[3];
     const uint64_t n = min(*n_arrived_dev, arrival_cap);
     const uint64_t a = (uint64_t)blockIdx.x * kBookThreads + threadIdx.x;
     if ((uint64_t)blockIdx.x * kBookThreads >= n) return;
     const uint64_t first_number = counters->n_arrived;
-    int stale = 0, invalid = 0;
+    bool stale = false, invalid = false;
     if (a < n) {
         const uint32_t slot = __ldg(&arrival[a]);
-        bool valid = false;
-        uint4 h0 = make_uint4(0, 0, 0, 0), h1 = h0;
-        if (slot < n_slots) {
-            const uint4* hp = reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(hdr_ring) + (uint64_t)slot * hdr_stride);
-            h0 = __ldg(hp);
-            h1 = __ldg(hp + 1);
-            const uint64_t off = (uint64_t)h1.x | ((uint64_t)h1.y << 32);
-            if (h1.z < W && h0.w < T) {
-                const uint64_t nt = __ldg(&numel[h0.w]);
-                if (off < nt && off % E == 0) {
-                    const uint64_t len = min((uint64_t)E, nt - off);
-                    valid = (h0.z == len * es) && (h0.x == __ldg(&chunkbase[h0.w]) + off / E);
-                }
-            }
-        }
+        const HeaderView h = validate_header(hdr_ring, hdr_stride, slot, n_slots, tensor_tab, T, W, E, es);
         uint32_t cell = kEmpty32;
-        if (!valid) invalid = 1;
-        else if (h0.y != round) stale = 1;
+        if (!h.valid) invalid = true;
+        else if (h.round != round) stale = true;
         else {
-            cell = (uint32_t)((uint64_t)h1.z * C + h0.x);
+            cell = (uint32_t)((uint64_t)h.worker * C + h.seq);
             atomicMin(&slot_key[cell], ((first_number + a) << 32) | slot);
         }
         cell_of[a] = cell;
     }
-    const int n_stale = __syncthreads_count(stale), n_inv = __syncthreads_count(invalid);
+    block_count3(false, stale, invalid, s_cnt);
     if (threadIdx.x == 0) {
-        if (n_stale) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_stale), (unsigned long long)n_stale);
-        if (n_inv) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_invalid), (unsigned long long)n_inv);
+        if (s_cnt[1]) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_stale), (unsigned long long)s_cnt[1]);
+        if (s_cnt[2]) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_invalid), (unsigned long long)s_cnt[2]);
     }
 }
 
@@ -335,68 +388,6 @@ __device__ __forceinline__ void st_agg16(float* p, float a, float b, float c, fl
     asm volatile("st.global.cs.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 
-template <int ES>
-__global__ void __launch_bounds__(kReduceThreads)
-k_reduce(const uint8_t* __restrict__ ring, const unsigned long long* __restrict__ slot_key,
-         const uint64_t* __restrict__ chunk_desc, float* __restrict__ agg, uint32_t W, uint32_t C, uint32_t P,
-         uint32_t VPC, int mean, float Wf)
-{
-    constexpr int VE = 16 / ES;            // elements per 16-byte vector: 4 fp32 or 8 bf16
-    const uint64_t i = (uint64_t)blockIdx.x * kReduceThreads + threadIdx.x;
-    if (i >= (uint64_t)C * VPC) return;
-    const uint32_t c = (uint32_t)(i / VPC), v = (uint32_t)(i - (uint64_t)c * VPC);
-    const uint64_t d = __ldg(&chunk_desc[c]);
-    const uint32_t len = (uint32_t)(d & 0xFFFFu), e0 = v * VE;
-    if (e0 >= len) return;
-
-    float acc[VE];
-#pragma unroll
-    for (int e = 0; e < VE; ++e) acc[e] = 0.0f;
-
-    const uint2* cell = reinterpret_cast<const uint2*>(slot_key) + c;   // low word = slot, all-ones = nothing arrived
-    for (uint32_t wb = 0; wb < W; wb += kWorkerBatch) {
-        uint32_t slot[kWorkerBatch];
-#pragma unroll
-        for (int k = 0; k < kWorkerBatch; ++k)
-            slot[k] = (wb + k < W) ? __ldg(&cell[(uint64_t)(wb + k) * C].x) : kEmpty32;
-        uint4 x[kWorkerBatch];
-#pragma unroll
-        for (int k = 0; k < kWorkerBatch; ++k)
-            if (slot[k] != kEmpty32) x[k] = ld_payload16(ring + (uint64_t)slot[k] * P + (uint64_t)v * 16);
-#pragma unroll
-        for (int k = 0; k < kWorkerBatch; ++k) {       // worker order: the additions are not reassociated
-            if (slot[k] == kEmpty32) continue;
-            if (ES == 4) {
-                acc[0] = __fadd_rn(acc[0], __uint_as_float(x[k].x));
-                acc[1] = __fadd_rn(acc[1], __uint_as_float(x[k].y));
-                acc[2] = __fadd_rn(acc[2], __uint_as_float(x[k].z));
-                acc[3] = __fadd_rn(acc[3], __uint_as_float(x[k].w));
-            } else {                                   // bf16 -> fp32 is a 16-bit shift
-                const uint32_t wd[4] = {x[k].x, x[k].y, x[k].z, x[k].w};
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    acc[2 * q] = __fadd_rn(acc[2 * q], __uint_as_float(wd[q] << 16));
-                    acc[2 * q + 1] = __fadd_rn(acc[2 * q + 1], __uint_as_float(wd[q] & 0xFFFF0000u));
-                }
-            }
-        }
-    }
-    if (mean) {
-#pragma unroll
-        for (int e = 0; e < VE; ++e) acc[e] = __fdiv_rn(acc[e], Wf);
-    }
-    float* out = agg + (d >> 16) + e0;
-    const uint32_t nv = min((uint32_t)VE, len - e0);
-    if (nv == VE && (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
-#pragma unroll
-        for (int q = 0; q < VE / 4; ++q) st_agg16(out + 4 * q, acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
-    } else {
-#pragma unroll
-        for (int e = 0; e < VE; ++e)
-            if (e < nv) out[e] = acc[e];
-    }
-}
-
 
 // ------------------------------------------------------------------------------------------------ tiled reduce
 // Persistent blocks walk over tiles of CH consecutive chunks.  For each tile the W x CH slot entries and the CH chunk
@@ -404,20 +395,23 @@ k_reduce(const uint8_t* __restrict__ ring, const unsigned long long* __restrict_
 // buffers), so the only global loads a thread waits for are the payload vectors themselves: WB * J independent
 // 128-bit loads per thread, issued together, then added in worker order.  A thread's J items are 256 vectors apart,
 // so every warp instruction touches 512 contiguous bytes of each payload it reads.
+//
+// Variants: J = 1 takes any worker count, WB workers per batch, accumulators kept across batches.  J > 1 is chosen
+// only for W <= WB (one batch): the J * WB loads are issued first and each item is then summed, finished and stored
+// on its own, so no more than one item's accumulators are live at a time and every variant fits the register budget
+// of four resident blocks per SM without spilling.
 #ifndef DBLP_REDUCE_THREADS
 #define DBLP_REDUCE_THREADS 256
 #endif
 #ifndef DBLP_REDUCE_MIN_BLOCKS
-#define DBLP_REDUCE_MIN_BLOCKS 4   // caps the one-item variant at 64 registers: four 256-thread blocks per SM
-#endif
-#ifndef DBLP_REDUCE_MIN_BLOCKS_WIDE
-#define DBLP_REDUCE_MIN_BLOCKS_WIDE 3   // resident blocks of the variants that hold 32 accumulators (bf16 with W <= 4, W = 1)
+#define DBLP_REDUCE_MIN_BLOCKS 4   // 64 registers: four 256-thread blocks per SM
 #endif
 #ifndef DBLP_REDUCE_J_WIDE
 #define DBLP_REDUCE_J_WIDE 1      // items per thread when W > 4 (8 workers per batch)
 #endif
 constexpr int kTileThreads = DBLP_REDUCE_THREADS;
 constexpr int kJWide = DBLP_REDUCE_J_WIDE;
+constexpr size_t kNormSmem = (kTileThreads / 32) * sizeof(double);   // static shared memory of the tiled kernels
 
 __device__ __forceinline__ void cp_async4(void* smem, const void* gmem)
 {
@@ -452,8 +446,155 @@ __device__ __forceinline__ uint32_t bf16_rne(float f)
     return (b + 0x7FFFu + ((b >> 16) & 1u)) >> 16;
 }
 
+// acc += x, element by element, plain fp32 additions; bf16 -> fp32 is a 16-bit shift.
+template <int ES>
+__device__ __forceinline__ void add_vector(float (&acc)[16 / ES], const uint4& x)
+{
+    if constexpr (ES == 4) {
+        acc[0] = __fadd_rn(acc[0], __uint_as_float(x.x));
+        acc[1] = __fadd_rn(acc[1], __uint_as_float(x.y));
+        acc[2] = __fadd_rn(acc[2], __uint_as_float(x.z));
+        acc[3] = __fadd_rn(acc[3], __uint_as_float(x.w));
+    } else {
+        const uint32_t wd[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            acc[2 * q] = __fadd_rn(acc[2 * q], __uint_as_float(wd[q] << 16));
+            acc[2 * q + 1] = __fadd_rn(acc[2 * q + 1], __uint_as_float(wd[q] & 0xFFFF0000u));
+        }
+    }
+}
+
+// What follows the sum of one 16-byte vector (elements e0 .. e0 + VE of a chunk of len elements whose first flat element
+// is chunk_elem): the mean, the store (fp32 or bf16; 128-bit when whole and aligned, element-wise at ragged edges), and
+// the fused extras.  sq collects the thread's share of the sum of squares.
+template <int ES, bool EXTRA>
+__device__ __forceinline__ void finish_vector(float (&acc)[16 / ES], float* __restrict__ agg, uint64_t chunk_elem,
+                                              uint32_t e0, uint32_t len, int mean, float Wf, const ReduceExtras& ex,
+                                              double& sq)
+{
+    constexpr int VE = 16 / ES;
+    if (mean == 1) {
+#pragma unroll
+        for (int e = 0; e < VE; ++e) acc[e] = __fdiv_rn(acc[e], Wf);
+    } else if (mean == 2) {                    // W a power of two: times 1/W is the same rounding, and cheaper
+#pragma unroll
+        for (int e = 0; e < VE; ++e) acc[e] = __fmul_rn(acc[e], Wf);
+    }
+    float* out = agg + chunk_elem + e0;
+    const uint32_t nv = min((uint32_t)VE, len - e0);
+    if (EXTRA && ex.out_bf16) {
+        uint16_t* out16 = reinterpret_cast<uint16_t*>(agg) + chunk_elem + e0;
+        if (nv == VE && (reinterpret_cast<uintptr_t>(out16) & 7u) == 0) {
+#pragma unroll
+            for (int q = 0; q < VE / 4; ++q)
+                reinterpret_cast<uint2*>(out16)[q] = make_uint2(bf16_rne(acc[4 * q]) | (bf16_rne(acc[4 * q + 1]) << 16),
+                                                                bf16_rne(acc[4 * q + 2]) | (bf16_rne(acc[4 * q + 3]) << 16));
+        } else {
+#pragma unroll
+            for (int e = 0; e < VE; ++e)
+                if (e < (int)nv) out16[e] = (uint16_t)bf16_rne(acc[e]);
+        }
+    } else if (nv == VE && (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
+#pragma unroll
+        for (int q = 0; q < VE / 4; ++q) st_agg16(out + 4 * q, acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
+    } else {
+#pragma unroll
+        for (int e = 0; e < VE; ++e)
+            if (e < (int)nv) out[e] = acc[e];
+    }
+    if (EXTRA) {
+        if (ex.norm_partials) {
+#pragma unroll
+            for (int e = 0; e < VE; ++e)
+                if (e < (int)nv) sq = __dadd_rn(sq, __dmul_rn((double)acc[e], (double)acc[e]));
+        }
+        if (ex.params) {
+            float* w_out = ex.params + chunk_elem + e0;
+#pragma unroll
+            for (int e = 0; e < VE; ++e)
+                if (e < (int)nv) w_out[e] = __fsub_rn(w_out[e], __fmul_rn(ex.lr, acc[e]));
+        }
+    }
+}
+
+// The simple form: one thread per (chunk, vector), tables read from global memory.  Serves worker counts whose slot
+// entries do not fit in shared memory.
+template <int ES>
+__global__ void __launch_bounds__(kReduceThreads)
+k_reduce(const uint8_t* __restrict__ ring, const unsigned long long* __restrict__ slot_key,
+         const uint64_t* __restrict__ chunk_desc, float* __restrict__ agg, uint32_t W, uint32_t C, uint32_t P,
+         uint32_t VPC, int mean, float Wf)
+{
+    constexpr int VE = 16 / ES;            // elements per 16-byte vector: 4 fp32 or 8 bf16
+    const uint64_t i = (uint64_t)blockIdx.x * kReduceThreads + threadIdx.x;
+    if (i >= (uint64_t)C * VPC) return;
+    const uint32_t c = (uint32_t)(i / VPC), v = (uint32_t)(i - (uint64_t)c * VPC);
+    const uint64_t d = __ldg(&chunk_desc[c]);
+    const uint32_t len = (uint32_t)(d & 0xFFFFu);
+    if (v * VE >= len) return;
+
+    float acc[VE];
+#pragma unroll
+    for (int e = 0; e < VE; ++e) acc[e] = 0.0f;
+    const uint2* cell = reinterpret_cast<const uint2*>(slot_key) + c;   // low word = slot, all-ones = nothing arrived
+    const uint8_t* src = ring + (uint64_t)v * 16;
+    for (uint32_t wb = 0; wb < W; wb += kWorkerBatch) {
+        uint4 x[kWorkerBatch];
+        uint32_t have = 0;
+#pragma unroll
+        for (int k = 0; k < kWorkerBatch; ++k) {
+            const uint32_t slot = (wb + k < W) ? __ldg(&cell[(uint64_t)(wb + k) * C].x) : kEmpty32;
+            if (slot != kEmpty32) {
+                have |= 1u << k;
+                x[k] = ld_payload16(src + (uint64_t)slot * P);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < kWorkerBatch; ++k)         // worker order: the additions are not reassociated
+            if ((have >> k) & 1u) add_vector<ES>(acc, x[k]);
+    }
+    double unused = 0.0;
+    finish_vector<ES, false>(acc, agg, d >> 16, v * VE, len, mean, Wf, ReduceExtras{nullptr, nullptr, 0.0f, 0}, unused);
+}
+
+// The tile's share of the fused norm: shuffle tree inside each warp, warps added in order by thread 0.
+// s_norm has one entry per warp; the call contains the barrier that also protects the tile's table buffer.
+template <bool EXTRA>
+__device__ __forceinline__ void finish_tile(double sq, double* s_norm, const ReduceExtras& ex, uint32_t tile)
+{
+    const uint32_t tid = threadIdx.x;
+    if (EXTRA && ex.norm_partials) {
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) sq = __dadd_rn(sq, __shfl_xor_sync(0xFFFFFFFFu, sq, d));
+        if ((tid & 31) == 0) s_norm[tid >> 5] = sq;
+    }
+    __syncthreads();                      // the buffer is refilled by the prefetch of the next iteration
+    if (EXTRA && ex.norm_partials && tid == 0) {
+        double t = 0.0;
+        for (int k = 0; k < kTileThreads / 32; ++k) t = __dadd_rn(t, s_norm[k]);
+        ex.norm_partials[tile] = t;
+    }
+}
+
+// Brings tile `tile`'s slot entries ([chunk][worker], low words of the claim table) and chunk descriptors into
+// buffer `buf` of the block's shared memory; the caller commits the cp.async group.
+__device__ __forceinline__ void prefetch_tile(uint64_t* sdesc, uint32_t* sslot, const uint2* __restrict__ cells,
+                                              const uint64_t* __restrict__ chunk_desc, uint32_t tile, uint32_t buf,
+                                              uint32_t CH, uint32_t C, uint32_t W)
+{
+    const uint32_t tid = threadIdx.x;
+    const uint32_t c0 = tile * CH, nch = min(CH, C - c0);
+    uint32_t* dst = sslot + (size_t)buf * CH * W;
+    for (uint32_t k = tid; k < nch * W; k += kTileThreads) {
+        const uint32_t w = k / nch, cl = k - w * nch;               // consecutive threads: consecutive chunks of one worker
+        cp_async4(&dst[cl * W + w], &cells[(uint64_t)w * C + c0 + cl].x);
+    }
+    for (uint32_t k = tid; k < nch; k += kTileThreads) cp_async8(&sdesc[buf * CH + k], &chunk_desc[c0 + k]);
+}
+
 template <int ES, int WB, int J, bool EXTRA>
-__global__ void __launch_bounds__(kTileThreads, ((ES == 4 && J < 8) || J == 1 ? DBLP_REDUCE_MIN_BLOCKS : DBLP_REDUCE_MIN_BLOCKS_WIDE))
+__global__ void __launch_bounds__(kTileThreads, DBLP_REDUCE_MIN_BLOCKS)
 k_reduce_tiled(const uint8_t* __restrict__ ring, const unsigned long long* __restrict__ slot_key,
                const uint64_t* __restrict__ chunk_desc, float* __restrict__ agg, uint32_t W, uint32_t C, uint32_t P,
                uint32_t VPC, uint32_t CH, uint32_t n_tiles, int mean, float Wf, ReduceExtras ex)
@@ -466,23 +607,15 @@ k_reduce_tiled(const uint8_t* __restrict__ ring, const unsigned long long* __res
     const uint32_t tid = threadIdx.x;
     const uint2* cells = reinterpret_cast<const uint2*>(slot_key);
     const uint32_t vpc_magic = (uint32_t)((0x100000000ull + VPC - 1) / VPC);   // ceil(2^32 / VPC); unused for VPC = 1
-
-    auto prefetch = [&](uint32_t tile, uint32_t buf) {
-        const uint32_t c0 = tile * CH, nch = min(CH, C - c0);
-        uint32_t* dst = sslot + (size_t)buf * CH * W;
-        for (uint32_t k = tid; k < nch * W; k += kTileThreads) {
-            const uint32_t w = k / nch, cl = k - w * nch;               // consecutive threads: consecutive chunks of one worker
-            cp_async4(&dst[cl * W + w], &cells[(uint64_t)w * C + c0 + cl].x);
-        }
-        for (uint32_t k = tid; k < nch; k += kTileThreads) cp_async8(&sdesc[buf * CH + k], &chunk_desc[c0 + k]);
-    };
+    // i / VPC for i < CH * VPC: exact because the plan keeps CH * VPC * VPC <= 2^32
+    auto chunk_of = [&](uint32_t i) { return VPC == 1 ? i : __umulhi(i, vpc_magic); };
 
     uint32_t tile = blockIdx.x, buf = 0;
-    if (tile < n_tiles) prefetch(tile, 0);
+    if (tile < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, tile, 0, CH, C, W);
     cp_async_commit();
     for (; tile < n_tiles; tile += gridDim.x, buf ^= 1) {
         const uint32_t next = tile + gridDim.x;
-        if (next < n_tiles) prefetch(next, buf ^ 1);
+        if (next < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, next, buf ^ 1, CH, C, W);
         cp_async_commit();
         cp_async_wait<1>();                   // everything but the group just committed has landed
         __syncthreads();
@@ -492,117 +625,70 @@ k_reduce_tiled(const uint8_t* __restrict__ ring, const unsigned long long* __res
         const uint32_t* ts = sslot + (size_t)buf * CH * W;
         double sq = 0.0;                      // this thread's share of the tile's sum of squares
         for (uint32_t i0 = tid; i0 < nvec; i0 += kTileThreads * J) {
-            float acc[J][VE];
-            uint32_t cl[J], v[J], len[J];
-            uint64_t dst[J];
-            bool act[J];
+            if (J == 1) {
+                const uint32_t cl = chunk_of(i0), v = i0 - cl * VPC;
+                const uint64_t d = td[cl];
+                const uint32_t len = (uint32_t)(d & 0xFFFFu);
+                if (v * VE >= len) continue;
+                const uint32_t* my = ts + cl * W;
+                const uint8_t* src = ring + (uint64_t)v * 16;
+                float acc[VE];
 #pragma unroll
-            for (int j = 0; j < J; ++j) {
-                const uint32_t i = i0 + j * kTileThreads;
-                act[j] = i < nvec;
-                cl[j] = !act[j] ? 0 : ((J > 1 && J < 8) || VPC == 1) ? i / VPC : __umulhi(i, vpc_magic);   // i / VPC (exact for i < 2^32 / VPC)
-                v[j] = i - cl[j] * VPC;
-                const uint64_t d = td[cl[j]];
-                len[j] = (uint32_t)(d & 0xFFFFu);
-                dst[j] = d >> 16;
-                act[j] = act[j] && v[j] * VE < len[j];
+                for (int e = 0; e < VE; ++e) acc[e] = 0.0f;
+                for (uint32_t wb = 0; wb < W; wb += WB) {
+                    uint4 x[WB];
+                    uint32_t have = 0;
 #pragma unroll
-                for (int e = 0; e < VE; ++e) acc[j][e] = 0.0f;
-            }
-            for (uint32_t wb = 0; wb < W; wb += WB) {
-                uint32_t slot[J][WB];
-                uint4 x[J][WB];
-#pragma unroll
-                for (int j = 0; j < J; ++j)
-#pragma unroll
-                    for (int k = 0; k < WB; ++k)
-                        slot[j][k] = (act[j] && wb + k < W) ? ts[cl[j] * W + wb + k] : kEmpty32;
-#pragma unroll
-                for (int j = 0; j < J; ++j)
-#pragma unroll
-                    for (int k = 0; k < WB; ++k)
-                        if (slot[j][k] != kEmpty32) x[j][k] = ld_payload16(ring + (uint64_t)slot[j][k] * P + (uint64_t)v[j] * 16);
-#pragma unroll
-                for (int j = 0; j < J; ++j)
-#pragma unroll
-                    for (int k = 0; k < WB; ++k) {               // worker order: the additions are not reassociated
-                        if (slot[j][k] == kEmpty32) continue;
-                        if (ES == 4) {
-                            acc[j][0] = __fadd_rn(acc[j][0], __uint_as_float(x[j][k].x));
-                            acc[j][1] = __fadd_rn(acc[j][1], __uint_as_float(x[j][k].y));
-                            acc[j][2] = __fadd_rn(acc[j][2], __uint_as_float(x[j][k].z));
-                            acc[j][3] = __fadd_rn(acc[j][3], __uint_as_float(x[j][k].w));
-                        } else {
-                            const uint32_t wd[4] = {x[j][k].x, x[j][k].y, x[j][k].z, x[j][k].w};
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                acc[j][2 * q] = __fadd_rn(acc[j][2 * q], __uint_as_float(wd[q] << 16));
-                                acc[j][2 * q + 1] = __fadd_rn(acc[j][2 * q + 1], __uint_as_float(wd[q] & 0xFFFF0000u));
-                            }
+                    for (int k = 0; k < WB; ++k) {
+                        const uint32_t slot = (wb + k < W) ? my[wb + k] : kEmpty32;
+                        if (slot != kEmpty32) {
+                            have |= 1u << k;
+                            x[k] = ld_payload16(src + (uint64_t)slot * P);
                         }
                     }
-            }
 #pragma unroll
-            for (int j = 0; j < J; ++j) {
-                if (!act[j]) continue;
-                if (mean == 1) {
-#pragma unroll
-                    for (int e = 0; e < VE; ++e) acc[j][e] = __fdiv_rn(acc[j][e], Wf);
-                } else if (mean == 2) {                    // W a power of two: times 1/W is the same rounding, and cheaper
-#pragma unroll
-                    for (int e = 0; e < VE; ++e) acc[j][e] = __fmul_rn(acc[j][e], Wf);
+                    for (int k = 0; k < WB; ++k)                     // worker order: the additions are not reassociated
+                        if ((have >> k) & 1u) add_vector<ES>(acc, x[k]);
                 }
-                const uint32_t e0 = v[j] * VE;
-                float* out = agg + dst[j] + e0;
-                const uint32_t nv = min((uint32_t)VE, len[j] - e0);
-                if (EXTRA && ex.out_bf16) {
-                    uint16_t* out16 = reinterpret_cast<uint16_t*>(agg) + dst[j] + e0;
-                    if (nv == VE && (reinterpret_cast<uintptr_t>(out16) & 7u) == 0) {
+                finish_vector<ES, EXTRA>(acc, agg, d >> 16, v * VE, len, mean, Wf, ex, sq);
+            } else {
+                uint4 x[J][WB];
+                uint32_t have = 0, act = 0;       // bit j * WB + k: worker k's packet of item j arrived; bit j: item j has data
 #pragma unroll
-                        for (int q = 0; q < VE / 4; ++q)
-                            reinterpret_cast<uint2*>(out16)[q] =
-                                make_uint2(bf16_rne(acc[j][4 * q]) | (bf16_rne(acc[j][4 * q + 1]) << 16),
-                                           bf16_rne(acc[j][4 * q + 2]) | (bf16_rne(acc[j][4 * q + 3]) << 16));
-                    } else {
+                for (int j = 0; j < J; ++j) {
+                    const uint32_t i = i0 + j * kTileThreads;
+                    if (i >= nvec) continue;
+                    const uint32_t cl = chunk_of(i), v = i - cl * VPC;
+                    if (v * VE >= (uint32_t)(td[cl] & 0xFFFFu)) continue;
+                    act |= 1u << j;
+                    const uint32_t* my = ts + cl * W;
+                    const uint8_t* src = ring + (uint64_t)v * 16;
 #pragma unroll
-                        for (int e = 0; e < VE; ++e)
-                            if (e < (int)nv) out16[e] = (uint16_t)bf16_rne(acc[j][e]);
+                    for (int k = 0; k < WB; ++k) {
+                        const uint32_t slot = ((uint32_t)k < W) ? my[k] : kEmpty32;
+                        if (slot != kEmpty32) {
+                            have |= 1u << (j * WB + k);
+                            x[j][k] = ld_payload16(src + (uint64_t)slot * P);
+                        }
                     }
-                } else if (nv == VE && (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
-#pragma unroll
-                    for (int q = 0; q < VE / 4; ++q)
-                        st_agg16(out + 4 * q, acc[j][4 * q], acc[j][4 * q + 1], acc[j][4 * q + 2], acc[j][4 * q + 3]);
-                } else {
-#pragma unroll
-                    for (int e = 0; e < VE; ++e)
-                        if (e < (int)nv) out[e] = acc[j][e];
                 }
-                if (EXTRA) {
-                    if (ex.norm_partials) {
 #pragma unroll
-                        for (int e = 0; e < VE; ++e)
-                            if (e < (int)nv) sq = __dadd_rn(sq, __dmul_rn((double)acc[j][e], (double)acc[j][e]));
-                    }
-                    if (ex.params) {
-                        float* w_out = ex.params + dst[j] + e0;
+                for (int j = 0; j < J; ++j) {
+                    if (!((act >> j) & 1u)) continue;
+                    float acc[VE];
 #pragma unroll
-                        for (int e = 0; e < VE; ++e)
-                            if (e < (int)nv) w_out[e] = __fsub_rn(w_out[e], __fmul_rn(ex.lr, acc[j][e]));
-                    }
+                    for (int e = 0; e < VE; ++e) acc[e] = 0.0f;
+#pragma unroll
+                    for (int k = 0; k < WB; ++k)                     // worker order
+                        if ((have >> (j * WB + k)) & 1u) add_vector<ES>(acc, x[j][k]);
+                    const uint32_t i = i0 + j * kTileThreads;
+                    const uint32_t cl = chunk_of(i), v = i - cl * VPC;
+                    const uint64_t d = td[cl];
+                    finish_vector<ES, EXTRA>(acc, agg, d >> 16, v * VE, (uint32_t)(d & 0xFFFFu), mean, Wf, ex, sq);
                 }
             }
         }
-        if (EXTRA && ex.norm_partials) {
-#pragma unroll
-            for (int d = 16; d >= 1; d >>= 1) sq = __dadd_rn(sq, __shfl_xor_sync(0xFFFFFFFFu, sq, d));
-            if ((tid & 31) == 0) s_norm[tid >> 5] = sq;
-        }
-        __syncthreads();                      // the buffer is refilled by the prefetch of the next iteration
-        if (EXTRA && ex.norm_partials && tid == 0) {
-            double t = 0.0;
-            for (int k = 0; k < kTileThreads / 32; ++k) t = __dadd_rn(t, s_norm[k]);
-            ex.norm_partials[tile] = t;
-        }
+        finish_tile<EXTRA>(sq, s_norm, ex, tile);
     }
     cp_async_wait<0>();
 }
@@ -611,9 +697,9 @@ k_reduce_tiled(const uint8_t* __restrict__ ring, const unsigned long long* __res
 // Same tiles, same tables in shared memory, same arithmetic as k_reduce_tiled, but a warp owns a whole chunk: its
 // descriptor and its W slot entries are read once per chunk (they are the same for all lanes), lane l handles the
 // vectors l, l + 32, ... of the chunk, S of them at a time, so that WB * S = 8 payload loads are in flight per thread
-// with almost no index arithmetic per load.
+// with almost no index arithmetic per load.  S > 1 only with W <= WB, as for the items of k_reduce_tiled.
 template <int ES, int WB, int S, bool EXTRA>
-__global__ void __launch_bounds__(kTileThreads, (S == 1 || (ES == 4 && S < 8)) ? DBLP_REDUCE_MIN_BLOCKS : DBLP_REDUCE_MIN_BLOCKS_WIDE)
+__global__ void __launch_bounds__(kTileThreads, (EXTRA && ES == 2 && S == 8) ? 3 : DBLP_REDUCE_MIN_BLOCKS)   // the one shape that needs more than 64 registers
 k_reduce_rows(const uint8_t* __restrict__ ring, const unsigned long long* __restrict__ slot_key,
               const uint64_t* __restrict__ chunk_desc, float* __restrict__ agg, uint32_t W, uint32_t C, uint32_t P,
               uint32_t CH, uint32_t n_tiles, int mean, float Wf, ReduceExtras ex)
@@ -627,22 +713,12 @@ k_reduce_rows(const uint8_t* __restrict__ ring, const unsigned long long* __rest
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint2* cells = reinterpret_cast<const uint2*>(slot_key);
 
-    auto prefetch = [&](uint32_t tile, uint32_t buf) {
-        const uint32_t c0 = tile * CH, nch = min(CH, C - c0);
-        uint32_t* dst = sslot + (size_t)buf * CH * W;
-        for (uint32_t k = tid; k < nch * W; k += kTileThreads) {
-            const uint32_t w = k / nch, cl = k - w * nch;
-            cp_async4(&dst[cl * W + w], &cells[(uint64_t)w * C + c0 + cl].x);
-        }
-        for (uint32_t k = tid; k < nch; k += kTileThreads) cp_async8(&sdesc[buf * CH + k], &chunk_desc[c0 + k]);
-    };
-
     uint32_t tile = blockIdx.x, buf = 0;
-    if (tile < n_tiles) prefetch(tile, 0);
+    if (tile < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, tile, 0, CH, C, W);
     cp_async_commit();
     for (; tile < n_tiles; tile += gridDim.x, buf ^= 1) {
         const uint32_t next = tile + gridDim.x;
-        if (next < n_tiles) prefetch(next, buf ^ 1);
+        if (next < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, next, buf ^ 1, CH, C, W);
         cp_async_commit();
         cp_async_wait<1>();
         __syncthreads();
@@ -655,111 +731,58 @@ k_reduce_rows(const uint8_t* __restrict__ ring, const unsigned long long* __rest
             const uint64_t d = td[cl];
             const uint32_t len = (uint32_t)(d & 0xFFFFu);
             const uint32_t nvc = (len + VE - 1) / VE;                    // vectors that hold data
-            float* const out_row = agg + (d >> 16);
+            const uint32_t* my = ts + cl * W;
             for (uint32_t vb = 0; vb < nvc; vb += 32 * S) {
-                float acc[S][VE];
+                const uint8_t* src = ring + (uint64_t)(vb + lane) * 16;
+                if (S == 1) {
+                    if (vb + lane >= nvc) continue;
+                    float acc[VE];
 #pragma unroll
-                for (int s = 0; s < S; ++s)
+                    for (int e = 0; e < VE; ++e) acc[e] = 0.0f;
+                    for (uint32_t wb = 0; wb < W; wb += WB) {
+                        uint4 x[WB];
+                        uint32_t have = 0;
 #pragma unroll
-                    for (int e = 0; e < VE; ++e) acc[s][e] = 0.0f;
-                for (uint32_t wb = 0; wb < W; wb += WB) {
-                    uint32_t slot[WB];
-                    uint4 x[S][WB];
-#pragma unroll
-                    for (int k = 0; k < WB; ++k) slot[k] = (wb + k < W) ? ts[cl * W + wb + k] : kEmpty32;
-#pragma unroll
-                    for (int k = 0; k < WB; ++k) {
-                        if (slot[k] == kEmpty32) continue;             // the same for the whole warp
-                        const uint8_t* src = ring + (uint64_t)slot[k] * P + (uint64_t)(vb + lane) * 16;
-#pragma unroll
-                        for (int s = 0; s < S; ++s)
-                            if (vb + lane + 32 * s < nvc) x[s][k] = ld_payload16(src + 512 * s);
-                    }
-#pragma unroll
-                    for (int k = 0; k < WB; ++k) {                      // worker order: the additions are not reassociated
-                        if (slot[k] == kEmpty32) continue;
-#pragma unroll
-                        for (int s = 0; s < S; ++s) {
-                            if (vb + lane + 32 * s >= nvc) continue;
-                            if (ES == 4) {
-                                acc[s][0] = __fadd_rn(acc[s][0], __uint_as_float(x[s][k].x));
-                                acc[s][1] = __fadd_rn(acc[s][1], __uint_as_float(x[s][k].y));
-                                acc[s][2] = __fadd_rn(acc[s][2], __uint_as_float(x[s][k].z));
-                                acc[s][3] = __fadd_rn(acc[s][3], __uint_as_float(x[s][k].w));
-                            } else {
-                                const uint32_t wd[4] = {x[s][k].x, x[s][k].y, x[s][k].z, x[s][k].w};
-#pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    acc[s][2 * q] = __fadd_rn(acc[s][2 * q], __uint_as_float(wd[q] << 16));
-                                    acc[s][2 * q + 1] = __fadd_rn(acc[s][2 * q + 1], __uint_as_float(wd[q] & 0xFFFF0000u));
-                                }
+                        for (int k = 0; k < WB; ++k) {
+                            const uint32_t slot = (wb + k < W) ? my[wb + k] : kEmpty32;   // the same for the whole warp
+                            if (slot != kEmpty32) {
+                                have |= 1u << k;
+                                x[k] = ld_payload16(src + (uint64_t)slot * P);
                             }
                         }
+#pragma unroll
+                        for (int k = 0; k < WB; ++k)                 // worker order: the additions are not reassociated
+                            if ((have >> k) & 1u) add_vector<ES>(acc, x[k]);
                     }
-                }
+                    finish_vector<ES, EXTRA>(acc, agg, d >> 16, (vb + lane) * VE, len, mean, Wf, ex, sq);
+                } else {
+                    uint4 x[S][WB];
+                    uint32_t have = 0;
 #pragma unroll
-                for (int s = 0; s < S; ++s) {
-                    const uint32_t v = vb + lane + 32 * s;
-                    if (v >= nvc) continue;
-                    if (mean == 1) {
+                    for (int k = 0; k < WB; ++k) {
+                        const uint32_t slot = ((uint32_t)k < W) ? my[k] : kEmpty32;
+                        if (slot == kEmpty32) continue;
+                        have |= 1u << k;
 #pragma unroll
-                        for (int e = 0; e < VE; ++e) acc[s][e] = __fdiv_rn(acc[s][e], Wf);
-                    } else if (mean == 2) {                // W a power of two: times 1/W is the same rounding, and cheaper
-#pragma unroll
-                        for (int e = 0; e < VE; ++e) acc[s][e] = __fmul_rn(acc[s][e], Wf);
+                        for (int q = 0; q < S; ++q)
+                            if (vb + lane + 32 * q < nvc) x[q][k] = ld_payload16(src + (uint64_t)slot * P + 512 * q);
                     }
-                    const uint32_t e0 = v * VE;
-                    float* out = out_row + e0;
-                    const uint32_t nv = min((uint32_t)VE, len - e0);
-                    if (EXTRA && ex.out_bf16) {
-                        uint16_t* out16 = reinterpret_cast<uint16_t*>(agg) + (d >> 16) + e0;
-                        if (nv == VE && (reinterpret_cast<uintptr_t>(out16) & 7u) == 0) {
 #pragma unroll
-                            for (int q = 0; q < VE / 4; ++q)
-                                reinterpret_cast<uint2*>(out16)[q] =
-                                    make_uint2(bf16_rne(acc[s][4 * q]) | (bf16_rne(acc[s][4 * q + 1]) << 16),
-                                               bf16_rne(acc[s][4 * q + 2]) | (bf16_rne(acc[s][4 * q + 3]) << 16));
-                        } else {
+                    for (int q = 0; q < S; ++q) {
+                        const uint32_t v = vb + lane + 32 * q;
+                        if (v >= nvc) continue;
+                        float acc[VE];
 #pragma unroll
-                            for (int e = 0; e < VE; ++e)
-                                if (e < (int)nv) out16[e] = (uint16_t)bf16_rne(acc[s][e]);
-                        }
-                    } else if (nv == VE && (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
+                        for (int e = 0; e < VE; ++e) acc[e] = 0.0f;
 #pragma unroll
-                        for (int q = 0; q < VE / 4; ++q)
-                            st_agg16(out + 4 * q, acc[s][4 * q], acc[s][4 * q + 1], acc[s][4 * q + 2], acc[s][4 * q + 3]);
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < VE; ++e)
-                            if (e < (int)nv) out[e] = acc[s][e];
-                    }
-                    if (EXTRA) {
-                        if (ex.norm_partials) {
-#pragma unroll
-                            for (int e = 0; e < VE; ++e)
-                                if (e < (int)nv) sq = __dadd_rn(sq, __dmul_rn((double)acc[s][e], (double)acc[s][e]));
-                        }
-                        if (ex.params) {
-                            float* w_out = ex.params + (d >> 16) + e0;
-#pragma unroll
-                            for (int e = 0; e < VE; ++e)
-                                if (e < (int)nv) w_out[e] = __fsub_rn(w_out[e], __fmul_rn(ex.lr, acc[s][e]));
-                        }
+                        for (int k = 0; k < WB; ++k)                 // worker order
+                            if ((have >> k) & 1u) add_vector<ES>(acc, x[q][k]);
+                        finish_vector<ES, EXTRA>(acc, agg, d >> 16, v * VE, len, mean, Wf, ex, sq);
                     }
                 }
             }
         }
-        if (EXTRA && ex.norm_partials) {
-#pragma unroll
-            for (int dlt = 16; dlt >= 1; dlt >>= 1) sq = __dadd_rn(sq, __shfl_xor_sync(0xFFFFFFFFu, sq, dlt));
-            if (lane == 0) s_norm[warp] = sq;
-        }
-        __syncthreads();
-        if (EXTRA && ex.norm_partials && tid == 0) {
-            double t = 0.0;
-            for (uint32_t k = 0; k < kWarps; ++k) t = __dadd_rn(t, s_norm[k]);
-            ex.norm_partials[tile] = t;
-        }
+        finish_tile<EXTRA>(sq, s_norm, ex, tile);
     }
     cp_async_wait<0>();
 }
@@ -861,7 +884,7 @@ int configure_reduce(dblp_plan* p, uint32_t ch_override, uint32_t grid_override)
     const uint32_t want = (2u * kTileThreads * J + p->VPC - 1) / p->VPC;
     if (CH < want) CH = want;
     const size_t per_chunk = (size_t)2 * (8 + 4 * (size_t)W);
-    const size_t smem_cap = 48 * 1024;
+    const size_t smem_cap = 48 * 1024 - kNormSmem;        // static + dynamic shared memory share the 48 KiB default limit
     if (per_chunk > smem_cap) return DBLP_OK;              // slot entries of one chunk do not fit: simple kernel
     if (CH * per_chunk > smem_cap) CH = (uint32_t)(smem_cap / per_chunk);
     const uint64_t ch_div_cap = 0x100000000ull / ((uint64_t)p->VPC * p->VPC);   // keeps the kernel's multiply-high division exact
@@ -909,7 +932,7 @@ extern "C" int dblp_aggregate_claim(const dblp_plan_t* plan, const dblp_hdr_t* h
     const unsigned grid = (unsigned)((arrival_cap + kBookThreads - 1) / kBookThreads);
     k_book<<<grid, kBookThreads, 0, static_cast<cudaStream_t>(stream)>>>(
         hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, reinterpret_cast<unsigned long long*>(slot_key), counters,
-        plan->d_numel, plan->d_chunkbase, plan->T, plan->W, plan->C, plan->E, plan->es, plan->hdr_stride);
+        plan->d_tensor_tab, plan->T, plan->W, plan->C, plan->E, plan->es, plan->hdr_stride);
     DBLP_LAUNCHED();
     return DBLP_OK;
 }
@@ -921,7 +944,7 @@ extern "C" int dblp_aggregate_bitmap(const dblp_plan_t* plan, const uint64_t* sl
     const uint64_t cells = plan->row_words * 32 * plan->W;
     k_bitmap<<<(unsigned)((cells + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
         reinterpret_cast<const unsigned long long*>(slot_key), recv_bitmap, plan->W, plan->C, plan->row_words, n_arrived_dev,
-        arrival_cap, counters);
+        arrival_cap, counters, 1);
     DBLP_LAUNCHED();
     return DBLP_OK;
 }
@@ -972,7 +995,7 @@ extern "C" int dblp_aggregate_book_stop(const dblp_plan_t* plan, const dblp_hdr_
     if (arrival_cap > 0) {
         const unsigned grid = (unsigned)((arrival_cap + kBookThreads - 1) / kBookThreads);
         k_book_claim<<<grid, kBookThreads, 0, s>>>(hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, keys, counters,
-                                                   cell_of, plan->d_numel, plan->d_chunkbase, plan->T, plan->W, plan->C,
+                                                   cell_of, plan->d_tensor_tab, plan->T, plan->W, plan->C,
                                                    plan->E, plan->es, plan->hdr_stride);
         DBLP_LAUNCHED();
         k_stop_count<<<l.n_blocks, 256, plan->W * sizeof(uint32_t), s>>>(cell_of, keys, n_arrived_dev, arrival_cap, counters,
@@ -986,7 +1009,7 @@ extern "C" int dblp_aggregate_book_stop(const dblp_plan_t* plan, const dblp_hdr_
     }
     const uint64_t cells = plan->row_words * 32 * plan->W;
     k_bitmap<<<(unsigned)((cells + 255) / 256), 256, 0, s>>>(keys, recv_bitmap, plan->W, plan->C, plan->row_words,
-                                                           n_arrived_dev, arrival_cap, counters);
+                                                           n_arrived_dev, arrival_cap, counters, 0);   // k_stop_apply has counted
     DBLP_LAUNCHED();
     return DBLP_OK;
 }

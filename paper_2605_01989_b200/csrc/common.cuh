@@ -82,7 +82,8 @@ __device__ __forceinline__ uint4 draw(const DrawKey& k, uint64_t a, uint32_t str
 // The plan: immutable after creation.  Device tables:
 //   chunk_desc[c]   = (first element of chunk c in the flat gradient) << 16 | elements in the chunk
 //   chunk_tensor[c] = tensor the chunk belongs to
-//   numel[t], base[t] (first flat element of tensor t), chunkbase[t] (sequence number of its first chunk; [T] = C)
+//   tensor_tab[t]   = (numel low, numel high, sequence number of the tensor's first chunk, 0): what the integrity
+//                     check needs, in one 16-byte load;  base[t] = first flat element of tensor t
 //   bucket_bounds[0..B], bound_ppm[B] (staging for per-bucket tolerances), ticket (see k_bound)
 // The staging buffer and the ticket make a plan serve one dblp_check_bound at a time.
 struct dblp_plan {
@@ -92,16 +93,23 @@ struct dblp_plan {
     uint32_t hdr_stride, pay_stride, pay_off;
     int dtype, device;
     uint64_t C, N, M, row_words;
+    // A shard of a split server (dblp_plan_set_shard) covers sequence numbers seq_off .. seq_off + C - 1 of a worker
+    // stream of C_stream chunks; otherwise C_stream = C and seq_off = 0.  Only the loss process looks at these.
+    uint64_t C_stream, seq_off;
     std::vector<uint64_t> h_numel, h_base;
     std::vector<uint32_t> h_chunkbase;
-    uint64_t* d_numel;
+    uint4* d_tensor_tab;
     uint64_t* d_base;
-    uint32_t* d_chunkbase;
     uint64_t* d_chunk_desc;
     uint32_t* d_chunk_tensor;
     uint32_t* d_bucket_bounds;
     uint32_t* d_bound_ppm;
     uint32_t* d_ticket;     // "blocks finished" counter of k_bound; zero between launches
+    // Host-side resources of the whole-round calls (round.cu): a high-priority stream for the work that runs beside
+    // the two bandwidth-bound kernels, a stream for host-to-device copies, and the events that order them.  They make
+    // a plan serve one whole-round call at a time.
+    cudaStream_t side, copy;
+    cudaEvent_t ev_fork, ev_join, ev_claimed, ev_done, ev_copy[2];
     // launch shape of the masked reduce (configure_reduce): red_variant = items per thread of the tiled kernel,
     // 0 = the simple one-vector-per-thread kernel
     uint32_t red_variant, red_CH, red_tiles, red_grid, red_rows;
@@ -110,4 +118,7 @@ struct dblp_plan {
 
 namespace dblp {
 int configure_reduce(dblp_plan* p, uint32_t ch_override, uint32_t grid_override);
+// dblp_packetize for workers w0 .. w0 + nw - 1 only; grads[k] is worker (w0 + k)'s gradient.
+int packetize_workers(const dblp_plan* plan, const void* const* grads, uint32_t w0, uint32_t nw, uint32_t round,
+                      dblp_hdr_t* hdr_ring, void* payload_ring, cudaStream_t s);
 }

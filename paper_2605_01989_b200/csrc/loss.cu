@@ -32,12 +32,15 @@ struct LossParams {
 
 // ------------------------------------------------------------------------------------------------ memoryless kinds
 __global__ void __launch_bounds__(kLossThreads)
-k_loss_pointwise(LossParams m, DrawKey dk, uint32_t W, uint64_t C, uint64_t row_words,
+k_loss_pointwise(LossParams m, DrawKey dk, uint32_t W, uint64_t C, uint64_t row_words, uint64_t C_stream, uint64_t seq_off,
                  const uint32_t* __restrict__ sent, uint32_t* __restrict__ delivered)
 {
+    // C_stream, seq_off: the plan covers sequence numbers seq_off .. seq_off + C - 1 of a worker stream of C_stream
+    // chunks (a shard of a split server; C_stream = C and seq_off = 0 otherwise).  Draws and the burst window live in
+    // the stream's numbering, so every shard sees the packet fates of the unsplit round.
     __shared__ uint64_t s_window_start;
     if (m.kind == DBLP_LOSS_MICROBURST) {
-        if (threadIdx.x == 0) s_window_start = (uint64_t)draw(dk, 0, kStreamWindow).x % (C - m.window_len + 1);
+        if (threadIdx.x == 0) s_window_start = (uint64_t)draw(dk, 0, kStreamWindow).x % (C_stream - m.window_len + 1);
         __syncthreads();
     }
     const uint64_t i = (uint64_t)blockIdx.x * kLossThreads + threadIdx.x;   // (row, word, lane)
@@ -48,10 +51,11 @@ k_loss_pointwise(LossParams m, DrawKey dk, uint32_t W, uint64_t C, uint64_t row_
     bool alive = false;
     if (seq < C && (!sent || ((__ldg(&sent[(uint64_t)w * row_words + (seq >> 5)]) >> (seq & 31)) & 1u))) {
         uint64_t t = 0;
+        const uint64_t gseq = seq_off + seq;
         if (m.kind == DBLP_LOSS_IID) t = m.t_drop;
         else if (m.kind == DBLP_LOSS_MICROBURST)
-            t = (seq >= s_window_start && seq < s_window_start + m.window_len) ? m.t_drop_in : m.t_drop_out;
-        const uint32_t u = draw(dk, (uint64_t)w * C + seq, kStreamPacket).x;
+            t = (gseq >= s_window_start && gseq < s_window_start + m.window_len) ? m.t_drop_in : m.t_drop_out;
+        const uint32_t u = draw(dk, (uint64_t)w * C_stream + gseq, kStreamPacket).x;
         alive = !((uint64_t)u < t);
     }
     const uint32_t word = __ballot_sync(0xFFFFFFFFu, alive);
@@ -312,22 +316,47 @@ k_arrival_scatter(uint32_t M, const uint32_t* __restrict__ perm_flag, const uint
     arrival[pos] = pf & 0x7FFFFFFFu;
 }
 
+// dst row w = bits seq_off .. seq_off + C - 1 of src row w (rows of src_words / dst_words words; padding bits zero).
+__global__ void __launch_bounds__(256)
+k_bitmap_columns(const uint32_t* __restrict__ src, uint64_t src_words, uint32_t W, uint64_t seq_off, uint64_t C,
+                 uint32_t* __restrict__ dst, uint64_t dst_words)
+{
+    const uint64_t j = (uint64_t)blockIdx.x * 256 + threadIdx.x;
+    if (j >= dst_words * W) return;
+    const uint32_t w = (uint32_t)(j / dst_words);
+    const uint64_t k = j - (uint64_t)w * dst_words;
+    const uint64_t first = seq_off + k * 32;                      // stream number of this word's bit 0
+    const uint32_t* row = src + (uint64_t)w * src_words;
+    const uint64_t sw = first >> 5;
+    const uint32_t sh = (uint32_t)(first & 31);
+    uint32_t x = row[sw] >> sh;
+    if (sh && sw + 1 < src_words) x |= row[sw + 1] << (32 - sh);
+    const uint64_t left = C - k * 32;                              // bits of the row that remain from this word on
+    if (left < 32) x &= (1u << left) - 1u;
+    dst[j] = x;
+}
+
 struct WorkspaceLayout {
-    size_t perm_flag, block_count, ge_fn, ge_state, total;
+    size_t perm_flag, block_count, ge_fn, ge_state, ge_mask, total;
     uint32_t n_perm_blocks, n_ge_blocks;
+    uint64_t stream_words;      // bitmap words per row of the whole worker stream
+    bool shard;
 };
 
 static WorkspaceLayout layout(const dblp_plan* p)
 {
     WorkspaceLayout l{};
     auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    l.shard = p->C_stream != p->C;
+    l.stream_words = (p->C_stream + 31) / 32;
     l.n_perm_blocks = (uint32_t)((p->M + kPermThreads - 1) / kPermThreads);
-    l.n_ge_blocks = (uint32_t)((p->row_words * p->W + kGeWordsPerBlock - 1) / kGeWordsPerBlock);
+    l.n_ge_blocks = (uint32_t)((l.stream_words * p->W + kGeWordsPerBlock - 1) / kGeWordsPerBlock);
     l.perm_flag = 0;
     l.block_count = up(l.perm_flag + p->M * sizeof(uint32_t));
     l.ge_fn = up(l.block_count + (size_t)l.n_perm_blocks * sizeof(uint32_t));
     l.ge_state = up(l.ge_fn + l.n_ge_blocks);
-    l.total = up(l.ge_state + l.n_ge_blocks);
+    l.ge_mask = up(l.ge_state + l.n_ge_blocks);       // a shard's burst chain is run over the whole stream, then cut
+    l.total = l.shard ? up(l.ge_mask + l.stream_words * p->W * sizeof(uint32_t)) : l.ge_mask;
     return l;
 }
 
@@ -358,7 +387,10 @@ extern "C" int dblp_apply_loss_resend(const dblp_plan_t* plan, const dblp_loss_m
                  model->t_drop_good <= limit && model->t_drop_bad <= limit && model->t_drop_in <= limit &&
                  model->t_drop_out <= limit, DBLP_EINVAL, "apply_loss: thresholds must lie in [0, 2^32]");
     if (model->kind == DBLP_LOSS_MICROBURST)
-        DBLP_REQUIRE(model->window_len <= plan->C, DBLP_EINVAL, "apply_loss: window longer than a worker's stream");
+        DBLP_REQUIRE(model->window_len <= plan->C_stream, DBLP_EINVAL, "apply_loss: window longer than a worker's stream");
+    DBLP_REQUIRE(!(l.shard && sent_bits && model->kind == DBLP_LOSS_GE), DBLP_EINVAL,
+                 "apply_loss: a burst chain over a subset of sent packets needs the whole stream's send set, which a "
+                 "shard plan does not have");
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     uint8_t* base = static_cast<uint8_t*>(ws);
@@ -372,17 +404,25 @@ extern "C" int dblp_apply_loss_resend(const dblp_plan_t* plan, const dblp_loss_m
     DrawKey dk{make_uint2((uint32_t)seed, (uint32_t)(seed >> 32)), attempt << 8, round};
 
     if (model->kind == DBLP_LOSS_GE) {
-        k_ge_partial<<<l.n_ge_blocks, kGeThreads, 0, s>>>(m, dk, plan->W, plan->C, plan->row_words, sent_bits, ge_fn);
+        // the chain is sequential along the whole worker stream: a shard runs it over the stream and keeps its columns
+        uint32_t* chain_out = l.shard ? reinterpret_cast<uint32_t*>(base + l.ge_mask) : delivered_bits;
+        k_ge_partial<<<l.n_ge_blocks, kGeThreads, 0, s>>>(m, dk, plan->W, plan->C_stream, l.stream_words, sent_bits, ge_fn);
         DBLP_LAUNCHED();
         k_ge_block_states<<<1, kScanThreads, 0, s>>>(ge_fn, ge_state, l.n_ge_blocks);
         DBLP_LAUNCHED();
-        k_ge_apply<<<l.n_ge_blocks, kGeThreads, 0, s>>>(m, dk, plan->W, plan->C, plan->row_words, sent_bits, ge_state,
-                                                       delivered_bits);
+        k_ge_apply<<<l.n_ge_blocks, kGeThreads, 0, s>>>(m, dk, plan->W, plan->C_stream, l.stream_words, sent_bits, ge_state,
+                                                       chain_out);
         DBLP_LAUNCHED();
+        if (l.shard) {
+            const uint64_t words = plan->row_words * plan->W;
+            k_bitmap_columns<<<(unsigned)((words + 255) / 256), 256, 0, s>>>(chain_out, l.stream_words, plan->W, plan->seq_off,
+                                                                            plan->C, delivered_bits, plan->row_words);
+            DBLP_LAUNCHED();
+        }
     } else {
         const uint64_t threads = plan->row_words * 32 * plan->W;
         k_loss_pointwise<<<(unsigned)((threads + kLossThreads - 1) / kLossThreads), kLossThreads, 0, s>>>(
-            m, dk, plan->W, plan->C, plan->row_words, sent_bits, delivered_bits);
+            m, dk, plan->W, plan->C, plan->row_words, plan->C_stream, plan->seq_off, sent_bits, delivered_bits);
         DBLP_LAUNCHED();
     }
 
@@ -439,8 +479,7 @@ static __device__ __align__(256) unsigned char g_static_scratch[DBLP_STATIC_SCRA
 
 namespace dblp {
 constexpr int kMaxDevices = 64;
-static void* g_static_scratch_addr[kMaxDevices];          // device address of the array, per device; null = not set up
-static std::atomic<bool> g_static_scratch_ready[kMaxDevices];
+static std::atomic<void*> g_static_scratch_addr[kMaxDevices];   // device address of the array, per device; null = not looked up yet
 }  // namespace dblp
 
 extern "C" int dblp_apply_loss_static(const dblp_plan_t* plan, const dblp_loss_model_t* model, uint64_t seed,
@@ -458,14 +497,14 @@ extern "C" int dblp_apply_loss_static(const dblp_plan_t* plan, const dblp_loss_m
     DBLP_REQUIRE(device == plan->device, DBLP_EINVAL, "apply_loss_static: device %d is current, the plan lives on device %d",
                  device, plan->device);
     DBLP_REQUIRE(device >= 0 && device < kMaxDevices, DBLP_ECAPACITY, "apply_loss_static: device index %d not supported", device);
-    if (!g_static_scratch_ready[device].load(std::memory_order_acquire)) {
+    void* addr = g_static_scratch_addr[device].load(std::memory_order_acquire);
+    if (!addr) {
         // In host code the array's name is only a handle; the kernels need its address in this device's memory.
-        void* addr = nullptr;
+        // Threads that get here together all look up the same address and store the same value.
         DBLP_CUDA(cudaGetSymbolAddress(&addr, g_static_scratch));
         DBLP_REQUIRE(addr, DBLP_ECUDA, "apply_loss_static: the scratch symbol has no address on device %d", device);
-        g_static_scratch_addr[device] = addr;
-        g_static_scratch_ready[device].store(true, std::memory_order_release);
+        g_static_scratch_addr[device].store(addr, std::memory_order_release);
     }
-    return dblp_apply_loss(plan, model, seed, round, attempt, delivered_bits, arrival, n_arrived_dev,
-                           g_static_scratch_addr[device], (size_t)DBLP_STATIC_SCRATCH_BYTES, stream);
+    return dblp_apply_loss(plan, model, seed, round, attempt, delivered_bits, arrival, n_arrived_dev, addr,
+                           (size_t)DBLP_STATIC_SCRATCH_BYTES, stream);
 }

@@ -107,6 +107,29 @@ k_packetize(GradPtrs grads, uint32_t w0, uint32_t C, uint32_t VPC, uint32_t pay_
     }
 }
 
+int packetize_workers(const dblp_plan* plan, const void* const* grads, uint32_t w_first, uint32_t n_workers, uint32_t round,
+                      dblp_hdr_t* hdr_ring, void* payload_ring, cudaStream_t s)
+{
+    uint32_t CH = (4096u + plan->VPC - 1) / plan->VPC;          // about 64 KB of payload per block
+    if (CH > kPackMaxTile) CH = kPackMaxTile;
+    const uint64_t gx = (plan->C + CH - 1) / CH;
+    DBLP_REQUIRE(gx < (1ull << 31), DBLP_ECAPACITY, "packetize: grid too large");
+    for (uint32_t w0 = w_first; w0 < w_first + n_workers; w0 += kMaxWorkersPerLaunch) {
+        const uint32_t nw = min(kMaxWorkersPerLaunch, w_first + n_workers - w0);
+        GradPtrs gp{};
+        for (uint32_t k = 0; k < nw; ++k) gp.p[k] = grads[w0 - w_first + k];
+        dim3 grid((unsigned)gx, nw);
+        if (plan->es == 4)
+            k_packetize<4><<<grid, kPackThreads, 0, s>>>(gp, w0, (uint32_t)plan->C, plan->VPC, plan->pay_stride, plan->hdr_stride, CH, round,
+                plan->d_chunk_desc, plan->d_chunk_tensor, plan->d_base, hdr_ring, static_cast<uint8_t*>(payload_ring) + plan->pay_off);
+        else
+            k_packetize<2><<<grid, kPackThreads, 0, s>>>(gp, w0, (uint32_t)plan->C, plan->VPC, plan->pay_stride, plan->hdr_stride, CH, round,
+                plan->d_chunk_desc, plan->d_chunk_tensor, plan->d_base, hdr_ring, static_cast<uint8_t*>(payload_ring) + plan->pay_off);
+        DBLP_LAUNCHED();
+    }
+    return DBLP_OK;
+}
+
 }  // namespace dblp
 
 using namespace dblp;
@@ -121,23 +144,5 @@ extern "C" int dblp_packetize(const dblp_plan_t* plan, const void* const* grads,
         DBLP_REQUIRE((reinterpret_cast<uintptr_t>(grads[w]) % plan->es) == 0, DBLP_EALIGN,
                      "packetize: gradient of worker %u is not element-aligned", w);
     }
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    uint32_t CH = (4096u + plan->VPC - 1) / plan->VPC;          // about 64 KB of payload per block
-    if (CH > kPackMaxTile) CH = kPackMaxTile;
-    const uint64_t gx = (plan->C + CH - 1) / CH;
-    DBLP_REQUIRE(gx < (1ull << 31), DBLP_ECAPACITY, "packetize: grid too large");
-    for (uint32_t w0 = 0; w0 < plan->W; w0 += kMaxWorkersPerLaunch) {
-        const uint32_t nw = min(kMaxWorkersPerLaunch, plan->W - w0);
-        GradPtrs gp{};
-        for (uint32_t k = 0; k < nw; ++k) gp.p[k] = grads[w0 + k];
-        dim3 grid((unsigned)gx, nw);
-        if (plan->es == 4)
-            k_packetize<4><<<grid, kPackThreads, 0, s>>>(gp, w0, (uint32_t)plan->C, plan->VPC, plan->pay_stride, plan->hdr_stride, CH, round,
-                plan->d_chunk_desc, plan->d_chunk_tensor, plan->d_base, hdr_ring, static_cast<uint8_t*>(payload_ring) + plan->pay_off);
-        else
-            k_packetize<2><<<grid, kPackThreads, 0, s>>>(gp, w0, (uint32_t)plan->C, plan->VPC, plan->pay_stride, plan->hdr_stride, CH, round,
-                plan->d_chunk_desc, plan->d_chunk_tensor, plan->d_base, hdr_ring, static_cast<uint8_t*>(payload_ring) + plan->pay_off);
-        DBLP_LAUNCHED();
-    }
-    return DBLP_OK;
+    return packetize_workers(plan, grads, 0, plan->W, round, hdr_ring, payload_ring, static_cast<cudaStream_t>(stream));
 }

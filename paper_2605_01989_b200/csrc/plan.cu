@@ -23,14 +23,32 @@ void set_error(const char* fmt, ...)
 
 static void free_tables(dblp_plan* p)
 {
-    cudaFree(p->d_numel);
+    cudaFree(p->d_tensor_tab);
     cudaFree(p->d_base);
-    cudaFree(p->d_chunkbase);
     cudaFree(p->d_chunk_desc);
     cudaFree(p->d_chunk_tensor);
     cudaFree(p->d_bucket_bounds);
     cudaFree(p->d_bound_ppm);
     cudaFree(p->d_ticket);
+    if (p->side) cudaStreamDestroy(p->side);
+    if (p->copy) cudaStreamDestroy(p->copy);
+    cudaEvent_t* evs[] = {&p->ev_fork, &p->ev_join, &p->ev_claimed, &p->ev_done, &p->ev_copy[0], &p->ev_copy[1]};
+    for (cudaEvent_t* e : evs)
+        if (*e) cudaEventDestroy(*e);
+}
+
+// Streams and events of the whole-round calls.  The side stream gets the highest priority the device offers, so that
+// its short kernels are scheduled between the blocks of the long bandwidth-bound ones instead of behind them.
+static cudaError_t create_round_resources(dblp_plan* p)
+{
+    int least = 0, greatest = 0;
+    cudaError_t e = cudaDeviceGetStreamPriorityRange(&least, &greatest);
+    if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&p->side, cudaStreamNonBlocking, greatest);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->copy, cudaStreamNonBlocking);
+    cudaEvent_t* evs[] = {&p->ev_fork, &p->ev_join, &p->ev_claimed, &p->ev_done, &p->ev_copy[0], &p->ev_copy[1]};
+    for (cudaEvent_t* ev : evs)
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
+    return e;
 }
 
 template <typename T>
@@ -45,8 +63,8 @@ static cudaError_t upload(T** dst, const std::vector<T>& src)
 
 using namespace dblp;
 
-extern "C" int dblp_plan_create(const uint64_t* tensor_numel, uint32_t T, int dtype, uint32_t payload_bytes, uint32_t W,
-                                const uint64_t* bucket_seq_bounds, uint32_t B, dblp_plan_t** out)
+static int plan_create(const uint64_t* tensor_numel, uint32_t T, int dtype, uint32_t payload_bytes, uint32_t W,
+                       const uint64_t* bucket_seq_bounds, uint32_t B, dblp_plan_t** out)
 {
     DBLP_REQUIRE(tensor_numel && out && T > 0 && W > 0 && B > 0, DBLP_EINVAL, "plan: null argument or zero count");
     DBLP_REQUIRE(dtype == DBLP_F32 || dtype == DBLP_BF16, DBLP_EINVAL, "plan: unknown dtype %d", dtype);
@@ -57,38 +75,43 @@ extern "C" int dblp_plan_create(const uint64_t* tensor_numel, uint32_t T, int dt
 
     dblp_plan* p = new (std::nothrow) dblp_plan();
     DBLP_REQUIRE(p, DBLP_EINVAL, "plan: out of host memory");
+    struct Guard {              // frees a half-built plan on every early return and on exceptions
+        dblp_plan* p;
+        ~Guard() { if (p) { free_tables(p); delete p; } }
+    } guard{p};
     p->T = T; p->W = W; p->B = B; p->P = payload_bytes; p->dtype = dtype;
     p->es = dtype == DBLP_F32 ? 4 : 2;
     p->E = payload_bytes / p->es;
     p->VE = 16 / p->es;
     p->VPC = payload_bytes / 16;
     p->hdr_stride = 32; p->pay_stride = payload_bytes; p->pay_off = 0;
-    p->d_numel = p->d_base = nullptr; p->d_chunk_desc = nullptr;
-    p->d_chunkbase = p->d_chunk_tensor = p->d_bucket_bounds = p->d_bound_ppm = p->d_ticket = nullptr;
+    p->d_tensor_tab = nullptr; p->d_base = nullptr; p->d_chunk_desc = nullptr;
+    p->d_chunk_tensor = p->d_bucket_bounds = p->d_bound_ppm = p->d_ticket = nullptr;
+    p->side = p->copy = nullptr;
+    p->ev_fork = p->ev_join = p->ev_claimed = p->ev_done = p->ev_copy[0] = p->ev_copy[1] = nullptr;
 
     uint64_t base = 0, c = 0;
     p->h_numel.assign(tensor_numel, tensor_numel + T);
     p->h_base.resize(T);
     p->h_chunkbase.resize((size_t)T + 1);
     for (uint32_t t = 0; t < T; ++t) {
-        if (tensor_numel[t] == 0) { delete p; DBLP_REQUIRE(false, DBLP_EINVAL, "plan: tensor %u has no elements", t); }
+        DBLP_REQUIRE(tensor_numel[t] != 0, DBLP_EINVAL, "plan: tensor %u has no elements", t);
         p->h_base[t] = base;
         p->h_chunkbase[t] = (uint32_t)c;
         base += tensor_numel[t];
         c += (tensor_numel[t] + p->E - 1) / p->E;
-        if (base >= (1ull << 47) || c * W >= (1ull << 31)) {
-            delete p;
-            DBLP_REQUIRE(false, DBLP_ECAPACITY, "plan: W * C must stay below 2^31 packets and N below 2^47 elements");
-        }
+        DBLP_REQUIRE(base < (1ull << 47) && c * W < (1ull << 31), DBLP_ECAPACITY,
+                     "plan: W * C must stay below 2^31 packets and N below 2^47 elements");
     }
     p->h_chunkbase[T] = (uint32_t)c;
     p->C = c; p->N = base; p->M = c * W; p->row_words = (c + 31) / 32;
+    p->C_stream = c; p->seq_off = 0;
 
     std::vector<uint32_t> bounds((size_t)B + 1);
     if (bucket_seq_bounds) {
         bool ok = bucket_seq_bounds[0] == 0 && bucket_seq_bounds[B] == c;
         for (uint32_t b = 0; b < B && ok; ++b) ok = bucket_seq_bounds[b] <= bucket_seq_bounds[b + 1];
-        if (!ok) { delete p; DBLP_REQUIRE(false, DBLP_EINVAL, "plan: bucket bounds must ascend from 0 to C = %llu", (unsigned long long)c); }
+        DBLP_REQUIRE(ok, DBLP_EINVAL, "plan: bucket bounds must ascend from 0 to C = %llu", (unsigned long long)c);
         for (uint32_t b = 0; b <= B; ++b) bounds[b] = (uint32_t)bucket_seq_bounds[b];
     } else {
         bounds[0] = 0; bounds[1] = (uint32_t)c;
@@ -105,30 +128,37 @@ extern "C" int dblp_plan_create(const uint64_t* tensor_numel, uint32_t T, int dt
         }
     }
 
+    std::vector<uint4> tab(T);
+    for (uint32_t t = 0; t < T; ++t)
+        tab[t] = make_uint4((uint32_t)tensor_numel[t], (uint32_t)(tensor_numel[t] >> 32), p->h_chunkbase[t], 0u);
+
     cudaError_t e = cudaGetDevice(&p->device);
-    if (e == cudaSuccess) e = upload(&p->d_numel, p->h_numel);
+    if (e == cudaSuccess) e = upload(&p->d_tensor_tab, tab);
     if (e == cudaSuccess) e = upload(&p->d_base, p->h_base);
-    if (e == cudaSuccess) e = upload(&p->d_chunkbase, p->h_chunkbase);
     if (e == cudaSuccess) e = upload(&p->d_chunk_desc, desc);
     if (e == cudaSuccess) e = upload(&p->d_chunk_tensor, owner);
     if (e == cudaSuccess) e = upload(&p->d_bucket_bounds, bounds);
     if (e == cudaSuccess) e = cudaMalloc((void**)&p->d_bound_ppm, sizeof(uint32_t) * B);
     if (e == cudaSuccess) e = cudaMalloc((void**)&p->d_ticket, sizeof(uint32_t));
     if (e == cudaSuccess) e = cudaMemset(p->d_ticket, 0, sizeof(uint32_t));
-    if (e != cudaSuccess) {
-        set_error("plan: device table setup failed: %s", cudaGetErrorString(e));
-        free_tables(p);
-        delete p;
-        return DBLP_ECUDA;
-    }
+    if (e == cudaSuccess) e = create_round_resources(p);
+    DBLP_REQUIRE(e == cudaSuccess, DBLP_ECUDA, "plan: device table setup failed: %s", cudaGetErrorString(e));
     const int rc = configure_reduce(p, 0, 0);
-    if (rc != DBLP_OK) {
-        free_tables(p);
-        delete p;
-        return rc;
-    }
+    if (rc != DBLP_OK) return rc;
+    guard.p = nullptr;
     *out = p;
     return DBLP_OK;
+}
+
+extern "C" int dblp_plan_create(const uint64_t* tensor_numel, uint32_t T, int dtype, uint32_t payload_bytes, uint32_t W,
+                                const uint64_t* bucket_seq_bounds, uint32_t B, dblp_plan_t** out)
+{
+    try {                      // the host tables are std::vectors: running out of host memory must not cross the C ABI
+        return plan_create(tensor_numel, T, dtype, payload_bytes, W, bucket_seq_bounds, B, out);
+    } catch (...) {
+        set_error("plan: out of host memory while building the chunk tables");
+        return DBLP_ECAPACITY;
+    }
 }
 
 extern "C" int dblp_plan_set_wire_format(dblp_plan_t* plan, int format)
@@ -141,6 +171,18 @@ extern "C" int dblp_plan_set_wire_format(dblp_plan_t* plan, int format)
     } else {
         DBLP_REQUIRE(false, DBLP_EINVAL, "plan_set_wire_format: unknown format %d", format);
     }
+    return DBLP_OK;
+}
+
+extern "C" int dblp_plan_set_shard(dblp_plan_t* plan, uint64_t stream_chunks, uint64_t seq_offset)
+{
+    DBLP_REQUIRE(plan, DBLP_EINVAL, "plan_set_shard: null plan");
+    DBLP_REQUIRE(seq_offset <= stream_chunks && plan->C <= stream_chunks - seq_offset, DBLP_EINVAL,
+                 "plan_set_shard: chunks %llu .. %llu do not lie inside a stream of %llu",
+                 (unsigned long long)seq_offset, (unsigned long long)(seq_offset + plan->C), (unsigned long long)stream_chunks);
+    DBLP_REQUIRE(stream_chunks * plan->W < (1ull << 31), DBLP_ECAPACITY, "plan_set_shard: W * stream chunks must stay below 2^31");
+    plan->C_stream = stream_chunks;
+    plan->seq_off = seq_offset;
     return DBLP_OK;
 }
 
@@ -181,6 +223,9 @@ extern "C" int dblp_loss_model_from_rates(int kind, double mean_loss, double mea
                      "loss_model_from_rates: burst length must be >= 1 and loss within [0, 1]");
         const double p_bg = 1.0 / mean_burst_len;
         const double p_gb = mean_loss < 1.0 ? p_bg * mean_loss / (1.0 - mean_loss) : 1.0;
+        DBLP_REQUIRE(p_gb <= 1.0, DBLP_EINVAL,
+                     "loss_model_from_rates: a mean loss of %g cannot be reached with bursts of mean length %g "
+                     "(P(Good->Bad) would be %g)", mean_loss, mean_burst_len, p_gb);
         out->t_gb = thr(p_gb); out->t_bg = thr(p_bg); out->t_init_bad = thr(mean_loss);
         out->t_drop_good = 0; out->t_drop_bad = 1ull << 32;
         break;

@@ -83,6 +83,8 @@ class LossSpec:
             p_bg = 1.0 / self.mean_burst
             pi = self.mean_loss
             p_gb = p_bg * pi / (1.0 - pi) if pi < 1.0 else 1.0
+            if p_gb > 1.0:
+                raise ValueError("a mean loss of %g cannot be reached with bursts of mean length %g" % (pi, self.mean_burst))
             return {"t_gb": threshold(p_gb), "t_bg": threshold(p_bg), "t_init_bad": threshold(pi),
                     "t_drop_good": 0, "t_drop_bad": TWO32}
         if self.kind == "microburst":

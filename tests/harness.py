@@ -150,3 +150,59 @@ def compare_bound(g, op, bitmap, ppm, bucket_bounds=None):
     assert_bits_equal(ok, o[2], "ok flags")
     assert allok == o[3]
     return o
+
+
+def oracle_round(op, om, host_grads, seed, rnd):
+    """One whole round by the oracle: headers, payloads, delivered bitmap, arrival list, booked state."""
+    o_hdr, o_pay = op.packetize(host_grads, rnd)
+    o_del, _ = op.loss_mask(om, seed, rnd)
+    o_arr, o_n = op.arrival(o_del, seed, rnd)
+    st = op.book(o_hdr, o_arr, o_n, rnd, op.new_state())
+    return o_hdr, o_pay, o_del, o_arr, o_n, st
+
+
+def device_round_parity(work, rounds, bound_ppm, flags=dblp.DBLP_MEAN, marks=None):
+    """`rounds` consecutive whole rounds through dblp_round_device (the library's two-stream schedule, every buffer
+    reused from one round to the next), each compared with the oracle bit for bit: rings, delivered bitmap, arrival
+    list, received bitmap, slot table, counters, bound outputs and the aggregate."""
+    grads = wl.make_grads(work, DEV)
+    host = to_host(grads, work.dtype)
+    g = GpuRound(work)
+    op = orc.Plan(work.numel, work.elem_size, work.payload_bytes, work.W)
+    gm, om = models_for(work, op.C)
+    for k in range(rounds):
+        rnd = work.round + k
+        dblp.dblp_round_device(g.plan, grads, gm, work.seed, rnd, bound_ppm, flags, g.buf, marks)
+        torch.cuda.synchronize()
+        o_hdr, o_pay, o_del, o_arr, o_n, st = oracle_round(op, om, host, work.seed, rnd)
+        assert_bits_equal(hdr_np(g.buf["hdr_ring"]), o_hdr, "header ring, round %d" % rnd)
+        assert_bits_equal(g.buf["payload_ring"].cpu().numpy(), o_pay, "payload ring, round %d" % rnd)
+        assert g.n_arrived() == o_n
+        assert_bits_equal(u32(g.buf["delivered_bits"]).reshape(op.W, op.row_words), o_del, "delivered bitmap")
+        assert_bits_equal(u32(g.buf["arrival"])[:o_n], o_arr[:o_n], "arrival list")
+        compare_state(g, st, op)
+        assert_bits_equal(g.buf["agg"].cpu().numpy(), op.reduce(o_pay, st, mean=(flags == dblp.DBLP_MEAN)),
+                          "aggregate, round %d" % rnd)
+        W, B = op.W, 1
+        o = op.check_bound(st["bitmap"], bound_ppm)
+        assert_bits_equal(u32(g.buf["recv_cnt"]).reshape(W, B), o[0], "recv counts")
+        assert_bits_equal(u32(g.buf["missing_cnt"]).reshape(W, B), o[1], "missing counts")
+        assert_bits_equal(g.buf["ok"].cpu().numpy().reshape(W, B), o[2], "ok flags")
+        assert int(u32(g.buf["all_ok"])[0]) == o[3]
+    g.close()
+
+
+def compare_bound_outputs(g, op, bitmap, ppm, saved=None):
+    """Two-step check of the bound outputs that a whole-round call leaves in its buffers: called with g right after the
+    round, it returns a host copy; called later with that copy and the oracle's bitmap, it compares."""
+    if saved is None:
+        W, B = g.plan.W, g.plan.B
+        b = g.buf
+        return (u32(b["recv_cnt"]).reshape(W, B).copy(), u32(b["missing_cnt"]).reshape(W, B).copy(),
+                b["ok"].cpu().numpy().reshape(W, B).copy(), int(u32(b["all_ok"])[0]))
+    o = op.check_bound(bitmap, ppm)
+    assert_bits_equal(saved[0], o[0], "recv counts of the round")
+    assert_bits_equal(saved[1], o[1], "missing counts of the round")
+    assert_bits_equal(saved[2], o[2], "ok flags of the round")
+    assert saved[3] == o[3]
+    return o

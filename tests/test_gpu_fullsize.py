@@ -1,10 +1,13 @@
 """GPU parity at the full sizes of the BERT-large-shaped (bf16) and GPT-2-XL-shaped (fp32) workloads, in the launch
-configuration the bench uses.  All integer results (headers, delivered bitmap, arrival list, received bitmap, slot
+configuration the bench times: the whole round goes through dblp_round_device (the library's two-stream schedule).  All integer results (headers, delivered bitmap, arrival list, received bitmap, slot
 table, counters, bound decisions) are compared in full against the CPU oracle.  The payload ring and the fp32
 aggregate are too large for the host, so they are checked (a) on sampled elements that the oracle computes one by
 one from the workers' own values, and (b) in full on the device against properties that hold at any size: every
 payload slot equals the gradient slice its oracle header names (padding zero), and the aggregate equals the
-left-to-right fp32 sum over workers of (oracle mask ? g_w : 0), evaluated with elementwise torch ops."""
+left-to-right fp32 sum over workers of (oracle mask ? g_w : 0), for the sum and for the mean, evaluated with elementwise
+torch ops.  The sample always contains the places where a wrong chunk table would show: both ends of every tensor, every
+element of every tensor's short last chunk, and the first element of each chunk that lost a packet and of the chunk
+after it."""
 import numpy as np
 import pytest
 import torch
@@ -33,10 +36,9 @@ def _fullsize(work, n_samples=200000):
     rnd, seed = work.round, work.seed
     grads = wl.make_grads(work, H.DEV)
     g = H.GpuRound(work)
-    g.packetize(grads, rnd)
-    g.apply_loss(gm, seed, rnd)
-    g.aggregate(rnd, dblp.DBLP_SUM)
+    dblp.dblp_round_device(g.plan, grads, gm, seed, rnd, work.bounds_ppm[0], dblp.DBLP_SUM, g.buf)
     torch.cuda.synchronize()
+    first = H.compare_bound_outputs(g, op, None, work.bounds_ppm[0])     # as the round itself left them; checked below
 
     # ---- integer results, in full
     o_hdr = op.headers(rnd)
@@ -48,6 +50,7 @@ def _fullsize(work, n_samples=200000):
     H.assert_bits_equal(H.u32(g.buf["arrival"])[:o_n], o_arr[:o_n], "arrival list")
     st = op.book(o_hdr, o_arr, o_n, rnd, op.new_state())
     H.compare_state(g, st, op)
+    H.compare_bound_outputs(None, op, st["bitmap"], work.bounds_ppm[0], first)
     for ppm in work.bounds_ppm:
         H.compare_bound(g, op, st["bitmap"], ppm)
 
@@ -65,8 +68,15 @@ def _fullsize(work, n_samples=200000):
 
     # ---- aggregate on sampled elements, one by one by the oracle
     rng = np.random.default_rng(seed)
-    edges = np.concatenate([op.base.astype(np.int64), op.base.astype(np.int64) + op.numel.astype(np.int64) - 1])
-    elem = np.unique(np.concatenate([rng.integers(0, op.N, n_samples), edges, [0, op.N - 1]]))
+    base, numel = op.base.astype(np.int64), op.numel.astype(np.int64)
+    edges = np.concatenate([base, base + numel - 1])
+    tails = [np.arange(base[t] + (numel[t] // E) * E, base[t] + numel[t]) for t in range(op.T) if numel[t] % E]
+    chunk_first = np.concatenate([base[t] + np.arange(-(-int(numel[t]) // E), dtype=np.int64) * E for t in range(op.T)])
+    got_all = np.unpackbits(o_del.view(np.uint8).reshape(op.W, -1), axis=1, bitorder="little")[:, :op.C].all(axis=0)
+    lossy = np.flatnonzero(~got_all)                       # chunks that lost at least one worker's packet
+    after = np.minimum(lossy + 1, op.C - 1)
+    elem = np.unique(np.concatenate([rng.integers(0, op.N, n_samples), edges, [0, op.N - 1], chunk_first[lossy],
+                                     chunk_first[after]] + tails))
     idx = torch.from_numpy(elem).to(H.DEV)
     vals = torch.stack([x[idx] for x in grads])
     vals = vals.view(torch.int16).cpu().numpy().view(np.uint16) if es == 2 else vals.cpu().numpy()
@@ -77,7 +87,6 @@ def _fullsize(work, n_samples=200000):
                             "sampled aggregate (flags %d)" % flags)
 
     # ---- aggregate, in full, against the masked left-to-right sum built from the oracle's bitmap
-    g.reduce(dblp.DBLP_SUM)
     chunk_len = torch.from_numpy(np.concatenate([
         np.minimum(E, int(op.numel[t]) - np.arange(-(-int(op.numel[t]) // E), dtype=np.int64) * E)
         for t in range(op.T)])).to(H.DEV)
@@ -88,7 +97,11 @@ def _fullsize(work, n_samples=200000):
         m = _expand_mask(torch.from_numpy(bits[w]).to(H.DEV), chunk_len, op.N)
         acc += torch.where(m, grads[w].float(), zero)
         del m
+    g.reduce(dblp.DBLP_SUM)
     assert torch.equal(acc.view(torch.int32), g.buf["agg"].view(torch.int32)), "full aggregate vs masked sum"
+    g.reduce(dblp.DBLP_MEAN)
+    acc /= float(op.W)                                     # IEEE fp32 division, as the definition of the mean
+    assert torch.equal(acc.view(torch.int32), g.buf["agg"].view(torch.int32)), "full mean vs masked sum / W"
     loss = 1.0 - o_n / op.M
     g.close()
     return loss

@@ -306,6 +306,52 @@ def test_round_host_entry_point_matches_the_oracle():
     g.close()
 
 
+def test_round_device_schedule_on_the_resnet50_shaped_workload():
+    """The schedule the bench times (apply_loss beside packetize, bitmap + check_bound beside the reduce, on the plan's
+    side stream), three consecutive rounds with every buffer reused, against the oracle."""
+    H.device_round_parity(wl.config(1), rounds=3, bound_ppm=24000)
+
+
+@pytest.mark.parametrize("dtype,P,W,flags", [("bf16", 4096, 3, dblp.DBLP_SUM), ("f32", 1408, 9, dblp.DBLP_MEAN),
+                                              ("f32", 16, 2, dblp.DBLP_MEAN)])
+def test_round_device_schedule_small_shapes(dtype, P, W, flags):
+    numel = RAGGED if P != 16 else [37, 1, 8, 5, 4096]
+    H.device_round_parity(work(numel, dtype, P, W, wl.LossSpec("ge", 0.1, 5.0), 23), rounds=4, bound_ppm=100000,
+                          flags=flags)
+
+
+def test_round_device_records_the_stage_marks():
+    marks = dblp.RoundMarks()
+    H.device_round_parity(wl.config(0), rounds=2, bound_ppm=8000, marks=marks)
+    order = [("begin", "packetize_end"), ("loss_begin", "loss_end"), ("receive_begin", "claim_end"),
+             ("claim_end", "reduce_end"), ("bound_begin", "bound_end"), ("reduce_end", "end"), ("begin", "end")]
+    for a, b in order:
+        assert marks.ms(a, b) >= 0.0, (a, b)
+    assert marks.ms("begin", "end") > 0.0
+
+
+def test_send_and_receive_halves_equal_the_whole_round():
+    w = work(RAGGED, "f32", 1408, 5, wl.LossSpec("iid", 0.1), 77)
+    grads = wl.make_grads(w, H.DEV)
+    a, b = H.GpuRound(w), H.GpuRound(w)
+    gm, _ = H.models_for(w, a.plan.C)
+    dblp.dblp_round_device(a.plan, grads, gm, w.seed, 9, 50000, dblp.DBLP_MEAN, a.buf)
+    dblp.dblp_round_send(b.plan, grads, gm, w.seed, 9, b.buf)
+    dblp.dblp_round_receive(b.plan, 9, 50000, dblp.DBLP_MEAN, b.buf)
+    torch.cuda.synchronize()
+    for name in ("hdr_ring", "payload_ring", "delivered_bits", "recv_bitmap", "slot_key", "counters", "agg", "recv_cnt",
+                 "missing_cnt", "ok", "all_ok"):
+        assert torch.equal(a.buf[name].view(torch.uint8), b.buf[name].view(torch.uint8)), name
+    a.close()
+    b.close()
+
+
+@pytest.mark.parametrize("W,P", [(766, 16), (766, 64), (761, 48), (1500, 32), (6134, 16)])
+def test_worker_counts_at_the_shared_memory_limit_of_the_tiled_reduce(W, P):
+    """Worker counts whose slot entries for a tile land on or just under the 48 KiB shared-memory limit."""
+    H.full_round_parity(work([100, 7, 64, 333], "f32", P, W, wl.LossSpec("iid", 0.3), W, bounds=(0, 300000)))
+
+
 def test_argument_errors_are_reported_not_faulted():
     w = work(ALIGNED, "f32", 1024, 2, wl.LossSpec("iid", 0.1), 1)
     g = H.GpuRound(w)
@@ -368,4 +414,8 @@ def test_library_counts_its_launches():
     g.aggregate(1)
     g.check_bound(1000)
     assert dblp.dblp_launch_count() - n0 == 1 + 6 + 3 + 1
+    n0 = dblp.dblp_launch_count()
+    dblp.dblp_round_device(g.plan, wl.make_grads(w, H.DEV), gm, 1, 2, 1000, dblp.DBLP_SUM, g.buf)
+    assert dblp.dblp_launch_count() - n0 == 1 + 6 + 3 + 1
+    torch.cuda.synchronize()
     g.close()
