@@ -1,17 +1,24 @@
 #!/usr/bin/env python
 """Throughput of the DBLP receive path on synthetic gradients.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet50|flat|bert|gpt2xl|sweep] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload gpt2xl|bert|resnet50|flat|sweep] [--impl reference]
 
-One step = one communication round through the library: round_reset, packetize, apply_loss, aggregate (bookkeeping +
-masked reduce) and check_bound, on gradients already resident in device memory.  The metric is algorithmic bytes read
-plus written per step divided by the step time (GB/s).  Prints one JSON line.
+One step = one communication round through the library's whole-round call (dblp_round_device): round_reset,
+packetize, apply_loss, aggregate (bookkeeping + masked reduce) and check_bound on gradients already resident in device
+memory, in the library's two-stream schedule.
+
+The metric is the bounded-loss aggregate rate: algorithmic bytes read plus written by the aggregate path (bookkeeping,
+masked reduce, tolerance test) divided by the time of that path inside the step, in GB/s.  `ms_per_step` is the whole
+step and `step_GBps` the whole step's bytes over it.  With no --workload the headline is the GPT-2-XL-shaped workload
+(the largest that fits one GPU) and `per_config` carries the ResNet-50- and BERT-large-shaped ones.  Prints one JSON
+line.
 
 With --impl reference the same round is run by the plain CPU checker on the host cores (a reported baseline).
-Under torchrun (N > 1) every rank runs its own independent round on its own GPU (weak scaling); the per-worker loss
-counts are summed across ranks once per step, the only exchange the sharded path has.
+Under torchrun (N > 1) the server is split by offset range over the ranks (strong scaling): every rank runs the round
+on its own run of tensors, the per-worker loss counts are summed over the ranks and the aggregate ranges all-gathered.
 """
 import argparse
+import copy
 import json
 import os
 import statistics
@@ -19,6 +26,7 @@ import sys
 import threading
 import time
 
+import numpy as np
 import torch
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
@@ -29,8 +37,15 @@ from paper_2605_01989_b200 import workloads as wl  # noqa: E402
 
 METRIC = "bounded-loss aggregate GB/s (bytes read+written)"
 WORKLOADS = {"flat": 0, "resnet50": 1, "bert": 2, "gpt2xl": 3, "sweep": 4}
+HEADLINE, PER_CONFIG = "gpt2xl", ("resnet50", "bert")
+DEFAULT_STEPS = {"flat": 2000, "resnet50": 500, "bert": 100, "gpt2xl": 40, "sweep": 300}
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+
+# DRAM bytes (read + write) that ncu counted for one launch of the reduce kernel, as a ratio to the launch's
+# algorithmic bytes, from a capture of a sweep point of about 1 GB (the bench workloads are too large to capture);
+# `traffic` scales it to the launch that is timed here.  An entry is removed whenever its kernel changes.
+NCU_TRAFFIC = {}
 
 
 def measured_peak():
@@ -41,10 +56,9 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def byte_model(work, C, n_arrived, payload_recv_bytes):
+def byte_model(W, N, s, C, n_arrived, payload_recv_bytes):
     """Algorithmic bytes of each stage for one round (what the method has to move, not what a kernel happens to)."""
-    W, N, s, M = work.W, work.N, work.elem_size, work.W * C
-    R = n_arrived
+    M, R = W * C, n_arrived
     stages = {
         "packetize": 2 * W * N * s + 32 * M,                       # read gradients, write payloads + headers
         "apply_loss": M // 8 + 4 * R,                              # delivered bitmap + arrival list
@@ -52,8 +66,22 @@ def byte_model(work, C, n_arrived, payload_recv_bytes):
         "reduce": payload_recv_bytes + 4 * N + 4 * M + 8 * C,      # received payloads, aggregate, slot entries, chunk table
         "check_bound": M // 8,
     }
-    stages["total"] = sum(stages.values())
+    stages["aggregate_path"] = stages["book"] + stages["reduce"] + stages["check_bound"]
+    stages["total"] = stages["packetize"] + stages["apply_loss"] + stages["aggregate_path"]
     return stages
+
+
+def chunk_lengths(numel, E):
+    return np.concatenate([np.minimum(E, n - np.arange(-(-n // E), dtype=np.int64) * E) for n in numel])
+
+
+def reduce_kernel_name(work):
+    W, es = work.W, work.elem_size
+    if W > 6000:
+        return "k_reduce<%d>" % es
+    wb, j = (1, 8) if W == 1 else (2, 4) if W <= 2 else (4, 2) if W <= 4 else (8, 1)
+    kind = "k_reduce_rows" if W <= 4 and work.payload_bytes >= 2048 else "k_reduce_tiled"
+    return "%s<%d, %d, %d, false>" % (kind, es, wb, j)
 
 
 class ClockSampler:
@@ -116,372 +144,413 @@ def physical_gpu_index(local_index):
 
 
 # ----------------------------------------------------------------------------------------------------------------------
-def run_gpu(args):
+class Job:
+    """Process-wide state of a GPU run: rank, world, device, process group."""
+
+    def __init__(self):
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+        torch.cuda.set_device(self.local)
+        self.dev = "cuda:%d" % self.local
+        self.dist = None
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.init_process_group("nccl", device_id=torch.device(self.dev))
+            self.dist = dist
+
+    def barrier(self):
+        if self.dist is not None:
+            self.dist.barrier()
+
+    def max_over_ranks(self, x):
+        if self.dist is None:
+            return x
+        t = torch.tensor([x], device=self.dev, dtype=torch.float64)
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def sum_over_ranks(self, x):
+        if self.dist is None:
+            return x
+        t = torch.tensor([x], device=self.dev, dtype=torch.float64)
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.SUM)
+        return float(t.item())
+
+
+def measure(job, name, steps, warmup, full):
+    """Times `steps` rounds of workload `name` (after `warmup` untimed ones) and returns its record.  `full` adds the
+    legs that only the headline carries: end to end from host buffers, and the CPU baseline."""
     from paper_2605_01989_b200 import binding as dblp
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
-    torch.cuda.set_device(local)
-    dev = "cuda:%d" % local
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device(dev))
-
-    work = wl.config(WORKLOADS[args.workload])
-    if world > 1:
-        work.seed = work.seed + 100 * rank            # every rank is an independent server shard with its own workers
-    plan = dblp.Plan(work.numel, work.dtype, work.payload_bytes, work.W)
-    buf = plan.alloc_round(dev)
-    grads = wl.make_grads(work, dev)
-    model = dblp.loss_model(work.loss.kind, **work.loss.thresholds(plan.C))
-    bound = work.bounds_ppm[0]
     from paper_2605_01989_b200 import shard
+    dev, world, rank = job.dev, job.world, job.rank
+    work = wl.config(WORKLOADS[name])
+    specs = shard.shard_specs(work.numel, work.E, world)
+    spec = specs[rank]
+    bound = work.bounds_ppm[-1] if name == "gpt2xl" else work.bounds_ppm[0]
+    shard.set_peer_shape(work.W, dev)
+    n_local = spec.elem_hi - spec.elem_lo
+    runner = None
+    if not spec.empty:
+        # one contiguous buffer for all workers' gradients: the end-to-end leg copies into the same memory
+        grads_dev = torch.empty(work.W * n_local, dtype=torch.float32 if work.dtype == "f32" else torch.bfloat16, device=dev)
+        grads = wl.make_grads(work, dev, elem_range=(spec.elem_lo, spec.elem_hi) if world > 1 else None, out=grads_dev)
+        runner = shard.GpuShardRunner(work, spec, dev, grads=grads)
+        runner.grads_dev = grads_dev
+    torch.cuda.synchronize()
 
-    # The loss process and the arrival order do not depend on the gradients, so apply_loss (ALU-bound) runs on a side
-    # stream while packetize (HBM-bound) runs on the main one; bookkeeping joins the two.  --serial puts all on one.
-    side = None if args.serial else torch.cuda.Stream(priority=-1)   # high priority: its small kernels slot in between packetize blocks
-    fork = torch.cuda.Event()
-    join = torch.cuda.Event()
-    booked = torch.cuda.Event()
+    exchanged = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
 
-    def lossy_channel(rnd, ev):
-        dblp.dblp_round_reset(plan, buf["recv_bitmap"], buf["slot_key"], buf["counters"])
-        if ev: ev[6].record()
-        dblp.dblp_apply_loss(plan, model, work.seed, rnd, 0, buf["delivered_bits"], buf["arrival"], buf["n_arrived"],
-                             buf["ws"])
-        if ev: ev[7].record()
+    def step(rnd, marks=None, k=None):
+        res = shard.sharded_round(runner, specs, rnd, bound, gather=world > 1, marks=marks)
+        if k is not None:
+            exchanged[k].record()
+        return res
 
-    def step(rnd, ev=None):
-        if ev: ev[0].record()
-        if side is not None:
-            fork.record()
-            with torch.cuda.stream(side):
-                side.wait_event(fork)
-                lossy_channel(rnd, ev)
-                join.record()
-        dblp.dblp_packetize(plan, grads, rnd, buf["hdr_ring"], buf["payload_ring"])
-        if ev: ev[1].record()
-        if side is not None:
-            torch.cuda.current_stream().wait_event(join)
-        else:
-            lossy_channel(rnd, ev)
-        if ev: ev[2].record()
-        if side is None:
-            dblp.dblp_aggregate_book(plan, buf["hdr_ring"], plan.M, buf["arrival"], buf["n_arrived"], plan.M, rnd,
-                                     buf["recv_bitmap"], buf["slot_key"], buf["counters"])
-        else:
-            dblp.dblp_aggregate_claim(plan, buf["hdr_ring"], plan.M, buf["arrival"], buf["n_arrived"], plan.M, rnd,
-                                      buf["slot_key"], buf["counters"])
-        if ev: ev[3].record()
-        if side is not None:                           # bitmap and tolerance test need the claims only: beside the reduce
-            booked.record()
-            with torch.cuda.stream(side):
-                side.wait_event(booked)
-                if ev: ev[8].record()
-                dblp.dblp_aggregate_bitmap(plan, buf["slot_key"], buf["n_arrived"], plan.M, buf["recv_bitmap"],
-                                           buf["counters"])
-                dblp.dblp_check_bound(plan, buf["recv_bitmap"], bound, buf["recv_cnt"], buf["missing_cnt"], buf["ok"],
-                                      buf["all_ok"])
-                if ev: ev[5].record()
-                join.record()
-        dblp.dblp_aggregate_reduce(plan, buf["payload_ring"], buf["slot_key"], buf["agg"], dblp.DBLP_MEAN)
-        if ev: ev[4].record()
-        if side is not None:
-            torch.cuda.current_stream().wait_event(join)
-            if ev: ev[9].record()
-        else:
-            if ev: ev[8].record()
-            dblp.dblp_check_bound(plan, buf["recv_bitmap"], bound, buf["recv_cnt"], buf["missing_cnt"], buf["ok"],
-                                  buf["all_ok"])
-            if ev: ev[5].record()
-            if ev: ev[9].record()
-        if dist is not None:                           # the sharded path's one exchange: loss counts per worker
-            shard.exchange_counts(buf["recv_cnt"], buf["missing_cnt"])
-
-    for i in range(args.warmup):
+    for i in range(warmup):
         step(1 + i)
     torch.cuda.synchronize()
-    if dist is not None:
-        dist.barrier()
+    job.barrier()
 
-    K = args.steps
+    marks = [dblp.RoundMarks() for _ in range(steps)] if runner is not None else [None] * steps
     t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(physical_gpu_index(local))
-    graph = None
-    if args.graph:
-        # Launch-bound sizes: the step (both streams, fork and join included) is captured once into a CUDA graph and
-        # replayed, so the host issues one launch per step.  Every replay redoes all the work with the captured round
-        # number; the per-stage times then come from a short eager pass after the timed region.
-        assert dist is None, "--graph is a single-GPU mode"
-        graph = torch.cuda.CUDAGraph()
-        launches0 = dblp.dblp_launch_count()
-        with torch.cuda.graph(graph):
-            step(100)
-        launches_per_step = dblp.dblp_launch_count() - launches0
-        for _ in range(3):
-            graph.replay()
-        torch.cuda.synchronize()
-        sampler.start()
-        t_begin.record()
-        for k in range(K):
-            graph.replay()
-        t_end.record()
-        torch.cuda.synchronize()
-        clocks = sampler.stop()
-        launches = launches_per_step * K
-        Ke = min(K, 50)
-        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(10)] for _ in range(Ke)]
-        for k in range(Ke):
-            step(100, evs[k])
-        torch.cuda.synchronize()
+    sampler = ClockSampler(physical_gpu_index(job.local))
+    launches0 = dblp.dblp_launch_count()
+    torch.cuda.synchronize()
+    job.barrier()
+    sampler.start()
+    t_begin.record()
+    for k in range(steps):
+        last = step(100 + k, marks[k], k)
+    t_end.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    launches = dblp.dblp_launch_count() - launches0
+    job.barrier()
+    last_round = 100 + steps - 1
+    ms_step = job.max_over_ranks(t_begin.elapsed_time(t_end)) / steps
+
+    # realised loss of the last round -> algorithmic bytes of this rank's shard
+    if runner is not None:
+        plan, buf = runner.plan, runner.buf
+        n_arrived = int(buf["n_arrived"].item())
+        bm = buf["recv_bitmap"].cpu().numpy().view("uint32").reshape(plan.W, plan.row_words)
+        bits = np.unpackbits(bm.view(np.uint8), axis=1, bitorder="little")[:, :plan.C]
+        payload_recv = int((bits.astype(np.int64) * chunk_lengths(spec.numel, work.E)[None, :]).sum()) * work.elem_size
+        mine = byte_model(work.W, n_local, work.elem_size, plan.C, n_arrived, payload_recv)
+        stage = lambda a, b: sum(m.ms(a, b) for m in marks) / steps                                  # noqa: E731
+        stage_ms = {"packetize": stage("begin", "packetize_end"), "apply_loss": stage("loss_begin", "loss_end"),
+                    "book": stage("receive_begin", "claim_end"), "reduce": stage("claim_end", "reduce_end"),
+                    "check_bound": stage("bound_begin", "bound_end"), "aggregate_path": stage("receive_begin", "end")}
+        if world > 1:                                        # the split server's aggregate path ends with its exchanges
+            stage_ms["aggregate_path_with_exchange"] = sum(
+                m.events["receive_begin"].elapsed_time(e) for m, e in zip(marks, exchanged)) / steps
     else:
-        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(10)] for _ in range(K)]
-        launches0 = dblp.dblp_launch_count()
-        torch.cuda.synchronize()
-        sampler.start()
-        t_begin.record()
-        for k in range(K):
-            step(100 + k, evs[k])
-        t_end.record()
-        torch.cuda.synchronize()
-        clocks = sampler.stop()
-        launches = dblp.dblp_launch_count() - launches0
-    if dist is not None:
-        dist.barrier()
-    ms_total = t_begin.elapsed_time(t_end)
-    if dist is not None:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
-    ms_step = ms_total / K
+        mine = byte_model(work.W, 0, work.elem_size, 0, 0, 0)
+        stage_ms = {k: 0.0 for k in ("packetize", "apply_loss", "book", "reduce", "check_bound", "aggregate_path")}
+        n_arrived = 0
+    bytes_all = {k: int(job.sum_over_ranks(v)) for k, v in mine.items()}
+    agg_key = "aggregate_path_with_exchange" if world > 1 else "aggregate_path"
+    agg_ms = job.max_over_ranks(stage_ms[agg_key])
+    arrived_all = job.sum_over_ranks(n_arrived)
 
-    spans = {"packetize": (0, 1), "apply_loss": (6, 7), "book": (2, 3), "reduce": (3, 4), "check_bound": (8, 5)}
-    stage_ms = {n: sum(e[a].elapsed_time(e[b]) for e in evs) / len(evs) for n, (a, b) in spans.items()}
+    verified = None
+    if world == 1 and not job.args.no_verify:
+        verified = verify_last_round(work, runner, last_round, bound, last)
 
-    # realised loss of the last round -> algorithmic bytes
-    n_arrived = int(buf["n_arrived"].item())
-    bm = buf["recv_bitmap"].cpu().numpy().view("uint32").reshape(plan.W, plan.row_words)
-    import numpy as np
-    bits = np.unpackbits(bm.view(np.uint8), axis=1, bitorder="little")[:, :plan.C]
-    E = work.E
-    chunk_len = np.concatenate([np.minimum(E, n - np.arange(-(-n // E), dtype=np.int64) * E) for n in work.numel])
-    payload_recv = int((bits.astype(np.int64) * chunk_len[None, :]).sum()) * work.elem_size
-    bytes_ = byte_model(work, plan.C, n_arrived, payload_recv)
+    peak, peak_kind = measured_peak()
+    red_gbs = mine["reduce"] / stage_ms["reduce"] / 1e6 if stage_ms["reduce"] else 0.0
+    agg_gbs = bytes_all["aggregate_path"] / agg_ms / 1e6
+    kernel = reduce_kernel_name(work)
+    ncu = NCU_TRAFFIC.get(kernel)
+    rec = {
+        "metric": METRIC, "value": agg_gbs, "unit": "GB/s", "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "vs_baseline": None, "dtype": work.dtype, "data": "synthetic",
+        "config": {"workload": work.name, "W": work.W, "payload_bytes": work.payload_bytes, "tensors": len(work.numel),
+                   "elements_per_worker": work.N, "packets": work.W * specs[0].stream_chunks, "loss": work.loss.kind,
+                   "realised_loss": 1.0 - arrived_all / (work.W * specs[0].stream_chunks), "bound_ppm": bound,
+                   "reduce": "mean, fixed worker order", "launch": "dblp_round_device, eager",
+                   "streams": "the library's schedule: apply_loss beside packetize, bitmap + check_bound beside the reduce, on the plan's high-priority stream",
+                   "l2": "inputs per step (%.0f MB) exceed the 126 MB L2; no flush" % (bytes_all["total"] / 1e6)
+                         if bytes_all["total"] > 4 * 126e6 else
+                         "inputs per step (%.0f MB) do not exceed the L2 by much: L2-resident, launch-bound" % (bytes_all["total"] / 1e6),
+                   "parallelism": "server split by offset range over %d GPUs" % world if world > 1 else "1 GPU"},
+        "value_is": "aggregate path (bookkeeping + masked reduce + tolerance test): its bytes / its time inside the step",
+        "pct_of_nominal_8TBs": 100.0 * agg_gbs / NOMINAL_HBM_GBS / world,
+        "pct_of_%s_peak" % peak_kind: 100.0 * agg_gbs / peak / world,
+        "step_GBps": bytes_all["total"] / ms_step / 1e6,
+        "bytes_per_step": bytes_all, "stage_ms": stage_ms,
+        "aggregate_path": {"what": "bookkeeping + masked reduce + bound check only", "GBps": agg_gbs, "ms": agg_ms,
+                           "pct_of_nominal_8TBs": 100.0 * agg_gbs / NOMINAL_HBM_GBS / world,
+                           "pct_of_%s_peak" % peak_kind: 100.0 * agg_gbs / peak / world},
+        "roofline": {"kernel": kernel, "bound": "hbm", "achieved": red_gbs, "peak": peak, "peak_kind": peak_kind,
+                     "unit": "GB/s", "frac": red_gbs / peak,
+                     "traffic": ncu["dram_bytes_per_algorithmic_byte"] * mine["reduce"] if ncu else None,
+                     "traffic_source": ncu["source"] if ncu else None,
+                     "algorithmic_bytes_per_launch": mine["reduce"], "ms_per_launch": stage_ms["reduce"]},
+        "clocks": clocks, "gpu_launches": launches, "verified": verified,
+    }
+    if world > 1:
+        rec["scaling"] = "strong"
+        rec["per_rank"] = {"rank": rank, "elements": n_local, "bytes_per_step": mine}
 
-    # end to end from host memory: pinned gradients in, aggregate + counts out, every step
-    e2e = None
-    if not args.no_e2e and work.W * work.N * work.elem_size > (16 << 30):
-        e2e = {"skipped": "host copies of %.0f GB of gradients: run with a smaller workload" % (work.W * work.N * work.elem_size / 1e9)}
-    elif not args.no_e2e:
-        grads_host = [g.cpu().pin_memory() for g in grads]
-        grads_dev = torch.empty(work.W * work.N, dtype=plan.torch_dtype, device=dev)
-        agg_host = torch.empty(work.N, dtype=torch.float32).pin_memory()
-        cnt_host = torch.zeros(7, dtype=torch.int64).pin_memory()
-        small = [torch.zeros(work.W, dtype=torch.int32).pin_memory() for _ in range(2)]
-        ok_host = torch.zeros(work.W, dtype=torch.uint8).pin_memory()
-        all_host = torch.zeros(1, dtype=torch.int32).pin_memory()
-        Ke = min(K, args.e2e_steps)
+    if full:
+        rec["e2e"] = end_to_end(job, work, runner, bound, mine, steps) if not job.args.no_e2e else None
+        if rank == 0 and world == 1 and job.args.extras:
+            rec["round_loop"], rec["reduce_extras"] = side_sections(work, runner, bound)
+    if runner is not None:
+        runner.close()
+        del grads, grads_dev
+    torch.cuda.empty_cache()
+    return rec, work, bytes_all
 
-        def e2e_step(rnd):
-            dblp.dblp_round_host(plan, grads_host, model, work.seed, rnd, bound, dblp.DBLP_MEAN, buf, grads_dev,
-                                 agg_host, cnt_host, small[0], small[1], ok_host, all_host)
 
-        for i in range(3):
-            e2e_step(50 + i)
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        for k in range(Ke):
-            e2e_step(100 + k)
-        b.record()
-        torch.cuda.synchronize()
-        ms_e2e = a.elapsed_time(b) / Ke
-        if dist is not None:
-            t = torch.tensor([ms_e2e], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
-        e2e = {"value": world * bytes_["total"] / ms_e2e / 1e6, "unit": "GB/s", "ms_per_step": ms_e2e, "steps": Ke,
-               "h2d_bytes_per_step": work.W * work.N * work.elem_size,
-               "d2h_bytes_per_step": work.N * 4 + 56 + work.W * 9 + 4}
-        del grads_host, grads_dev
+def verify_last_round(work, runner, rnd, bound, result):
+    """Outside the timed region: the state the last timed round left on the device against the CPU checker -- arrival
+    count, received bitmap, all counters, the tolerance outputs, and a sample of aggregate elements (random ones, both
+    ends of every tensor, every tensor's short last chunk)."""
+    from oracle import dblp_oracle as orc
+    from paper_2605_01989_b200 import binding as dblp
+    t0 = time.perf_counter()
+    plan, buf = runner.plan, runner.buf
+    op = orc.Plan(work.numel, work.elem_size, work.payload_bytes, work.W)
+    om = orc.loss_model(work.loss.kind, **work.loss.thresholds(op.C))
+    o_del, _ = op.loss_mask(om, work.seed, rnd)
+    o_arr, o_n = op.arrival(o_del, work.seed, rnd)
+    st = op.book(op.headers(rnd), o_arr, o_n, rnd, op.new_state())
+    checks = {}
+    checks["n_arrived"] = int(buf["n_arrived"].item()) == o_n
+    checks["received_bitmap"] = buf["recv_bitmap"].cpu().numpy().view(np.uint32).tobytes() == st["bitmap"].tobytes()
+    c = dblp.counters_dict(buf["counters"])
+    checks["counters"] = {k: c[k] for k in dblp.COUNTER_FIELDS} == st["counters"].as_dict() and c["status"] == 0
+    recv, miss, ok, all_ok = op.check_bound(st["bitmap"], bound)
+    checks["bound_outputs"] = (buf["recv_cnt"].cpu().numpy().view(np.uint32).tolist() == recv[:, 0].tolist() and
+                               buf["missing_cnt"].cpu().numpy().view(np.uint32).tolist() == miss[:, 0].tolist() and
+                               buf["ok"].cpu().numpy().tolist() == ok[:, 0].tolist() and
+                               int(buf["all_ok"].item()) == all_ok)
+    from paper_2605_01989_b200 import shard
+    checks["decision"] = shard.decision(result, dblp.dblp_bound_ok, bound) == (ok[:, 0].tolist(), all_ok)
+    rng = np.random.default_rng(rnd)
+    base, numel, E = op.base.astype(np.int64), op.numel.astype(np.int64), op.E
+    tails = [np.arange(base[t] + (numel[t] // E) * E, base[t] + numel[t]) for t in range(op.T) if numel[t] % E]
+    elem = np.unique(np.concatenate([rng.integers(0, op.N, 100000), base, base + numel - 1] + tails))
+    idx = torch.from_numpy(elem).to(buf["agg"].device)
+    vals = torch.stack([x[idx] for x in runner.grads])
+    vals = vals.view(torch.int16).cpu().numpy().view(np.uint16) if work.elem_size == 2 else vals.cpu().numpy()
+    want = op.reduce_at(st["bitmap"], elem, vals, mean=True)
+    checks["aggregate_sample"] = buf["agg"][idx].cpu().numpy().tobytes() == want.tobytes()
+    return {"ok": all(checks.values()), "checks": checks, "round": rnd, "sampled_elements": int(len(elem)),
+            "seconds": time.perf_counter() - t0}
 
-    # the control loop under heavy i.i.d. bursts: attempts until every worker passes, low vs high tolerance
-    # (the mechanism behind the paper's latency tables; not part of the timed step)
-    round_loop = None
-    if rank == 0 and world == 1 and not args.no_round_loop:
-        p_low = bound
-        p_high = bound + 400000
-        round_loop = []
-        dblp.dblp_packetize(plan, grads, 7, buf["hdr_ring"], buf["payload_ring"])
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        for burst in (0.6, 0.7, 0.8, 0.9):
-            m = dblp.loss_model("iid", t_drop=wl.threshold(burst))
-            row = {"loss": burst}
-            for name, ppm in (("p_low", p_low), ("p_high", p_high)):
-                dblp.dblp_round_reset(plan, buf["recv_bitmap"], buf["slot_key"], buf["counters"])
-                a.record()
-                attempts, ok = dblp.dblp_round_until_stop(plan, m, work.seed, 7, ppm, 400, True, buf)
-                b.record()
-                torch.cuda.synchronize()
-                row[name] = {"ppm": ppm, "attempts": attempts, "all_ok": ok, "ms": a.elapsed_time(b)}
-            row["attempt_ratio"] = row["p_low"]["attempts"] / max(1, row["p_high"]["attempts"])
-            round_loop.append(row)
 
-    # the reduce with its fused extras (norm for Eq. 1, worker update), timed alone; not part of the timed step
-    extras = None
-    if rank == 0 and world == 1 and not args.no_round_loop:
-        dblp.dblp_round_reset(plan, buf["recv_bitmap"], buf["slot_key"], buf["counters"])
-        step(7)
-        scratch = torch.empty(max(1, dblp.dblp_norm_scratch_count(plan)), dtype=torch.float64, device=dev)
-        norm_out = torch.zeros(2, dtype=torch.float64, device=dev)
-        params = torch.zeros(work.N, dtype=torch.float32, device=dev)
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+def end_to_end(job, work, runner, bound, mine, steps):
+    """The same round through dblp_round_host: every step copies all workers' gradients from pinned host memory and
+    reads the aggregate, the counters and the tolerance outputs back."""
+    from paper_2605_01989_b200 import binding as dblp
+    if runner is None:
+        return None
+    dev = job.dev
+    plan, buf = runner.plan, runner.buf
+    n_local = runner.spec.elem_hi - runner.spec.elem_lo
+    dtype = runner.grads[0].dtype
+    pinned = True
+    try:
+        grads_host = [torch.empty(n_local, dtype=dtype, pin_memory=True) for _ in range(work.W)]
+        agg_host = torch.empty(n_local, dtype=torch.float32, pin_memory=True)
+    except RuntimeError:
+        pinned = False
+        grads_host = [torch.empty(n_local, dtype=dtype) for _ in range(work.W)]
+        agg_host = torch.empty(n_local, dtype=torch.float32)
+    for h, g in zip(grads_host, runner.grads):
+        h.copy_(g)
+    grads_dev = runner.grads_dev                  # the workers' gradients back to back: the copies land where they already are
+    cnt_host = torch.zeros(7, dtype=torch.int64).pin_memory()
+    small = [torch.zeros(work.W, dtype=torch.int32).pin_memory() for _ in range(2)]
+    ok_host = torch.zeros(work.W, dtype=torch.uint8).pin_memory()
+    all_host = torch.zeros(1, dtype=torch.int32).pin_memory()
+    h2d = work.W * n_local * work.elem_size
+    Ke = max(3, min(steps, job.args.e2e_steps, int(30e9 / max(1, h2d)) + 3))      # about half a minute of copies at most
 
-        def timed(fn, reps=50):
-            for _ in range(3):
-                fn()
+    def e2e_step(rnd):
+        dblp.dblp_round_host(plan, grads_host, runner.model, work.seed, rnd, bound, dblp.DBLP_MEAN, buf, grads_dev,
+                             agg_host, cnt_host, small[0], small[1], ok_host, all_host)
+
+    for i in range(3):
+        e2e_step(50 + i)
+    torch.cuda.synchronize()
+    job.barrier()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for k in range(Ke):
+        e2e_step(100 + k)
+    b.record()
+    torch.cuda.synchronize()
+    ms_e2e = job.max_over_ranks(a.elapsed_time(b) / Ke)
+    agg_bytes = job.sum_over_ranks(mine["aggregate_path"])
+    return {"value": agg_bytes / ms_e2e / 1e6, "unit": "GB/s", "ms_per_step": ms_e2e, "steps": Ke,
+            "what": "dblp_round_host: the metric's bytes over the whole call, host-to-device copies of all gradients and "
+                    "device-to-host copy of the aggregate included",
+            "step_GBps": job.sum_over_ranks(mine["total"]) / ms_e2e / 1e6,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": n_local * 4 + 56 + work.W * 9 + 4, "pinned": pinned,
+            "h2d_GBps": h2d / ms_e2e / 1e6}
+
+
+def side_sections(work, runner, bound):
+    """Untimed extras (--extras): the control loop under heavy loss (attempts until every worker passes, low against
+    high tolerance: the mechanism behind the paper's latency tables) and the reduce with its fused norm / update."""
+    from paper_2605_01989_b200 import binding as dblp
+    plan, buf, grads = runner.plan, runner.buf, runner.grads
+    p_low, p_high = bound, bound + 400000
+    round_loop = []
+    dblp.dblp_packetize(plan, grads, 7, buf["hdr_ring"], buf["payload_ring"])
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for burst in (0.6, 0.7, 0.8, 0.9):
+        m = dblp.loss_model("iid", t_drop=wl.threshold(burst))
+        row = {"loss": burst}
+        for name, ppm in (("p_low", p_low), ("p_high", p_high)):
+            dblp.dblp_round_reset(plan, buf["recv_bitmap"], buf["slot_key"], buf["counters"])
             a.record()
-            for _ in range(reps):
-                fn()
+            attempts, ok = dblp.dblp_round_until_stop(plan, m, work.seed, 7, ppm, 400, True, buf)
             b.record()
             torch.cuda.synchronize()
-            return a.elapsed_time(b) / reps
+            row[name] = {"ppm": ppm, "attempts": attempts, "all_ok": ok, "ms": a.elapsed_time(b)}
+        row["attempt_ratio"] = row["p_low"]["attempts"] / max(1, row["p_high"]["attempts"])
+        round_loop.append(row)
 
-        extras = {
-            "reduce_ms": timed(lambda: dblp.dblp_aggregate_reduce(plan, buf["payload_ring"], buf["slot_key"], buf["agg"],
-                                                                  dblp.DBLP_MEAN)),
-            "reduce_norm_ms": timed(lambda: dblp.dblp_aggregate_reduce_ex(plan, buf["payload_ring"], buf["slot_key"],
-                                                                          buf["agg"], dblp.DBLP_MEAN, scratch, norm_out)),
-            "reduce_norm_update_ms": timed(lambda: dblp.dblp_aggregate_reduce_ex(
-                plan, buf["payload_ring"], buf["slot_key"], buf["agg"], dblp.DBLP_MEAN, scratch, norm_out, params, 0.01)),
-            "reduce_atomic_order_free_ms": timed(lambda: dblp.dblp_aggregate_reduce_atomic(
-                plan, buf["payload_ring"], buf["slot_key"], buf["agg"], dblp.DBLP_MEAN)),
-            "grad_norm": float(norm_out[1].item()),
-        }
-        del scratch, params
+    dblp.dblp_round_device(plan, grads, runner.model, work.seed, 7, bound, dblp.DBLP_MEAN, buf)
+    dev = buf["agg"].device
+    scratch = torch.empty(max(1, dblp.dblp_norm_scratch_count(plan)), dtype=torch.float64, device=dev)
+    norm_out = torch.zeros(2, dtype=torch.float64, device=dev)
+    params = torch.zeros(plan.N, dtype=torch.float32, device=dev)
 
-    cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu = cpu_baseline(work, bytes_["total"])
+    def timed(fn, reps=20):
+        for _ in range(3):
+            fn()
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
 
-    if dist is not None:
-        dist.barrier()
-        dist.destroy_process_group()
-    if rank != 0:
-        return
-    peak, peak_kind = measured_peak()
-    red_gbs = bytes_["reduce"] / stage_ms["reduce"] / 1e6
-    agg_ms = sum(e[2].elapsed_time(e[9]) for e in evs) / len(evs)      # bookkeeping start to the end of reduce and bound check
-    agg_gbs = (bytes_["book"] + bytes_["reduce"] + bytes_["check_bound"]) / agg_ms / 1e6
-    out = {
-        "metric": METRIC, "value": world * bytes_["total"] / ms_step / 1e6, "unit": "GB/s", "n_gpus": world,
-        "steps": K, "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": work.dtype, "data": "synthetic",
-        "config": {"workload": work.name, "W": work.W, "payload_bytes": work.payload_bytes, "tensors": len(work.numel),
-                   "elements_per_worker": work.N, "packets": plan.M, "loss": work.loss.kind,
-                   "realised_loss": 1.0 - n_arrived / plan.M, "bound_ppm": bound, "reduce": "mean, fixed worker order",
-                   "launch": "CUDA graph replay" if graph is not None else "eager",
-                   "streams": "one" if side is None else "apply_loss beside packetize, bitmap + check_bound beside the reduce, on a high-priority side stream",
-                   "l2": "inputs per step (%.0f MB) exceed the 126 MB L2; no flush" % (bytes_["total"] / 1e6),
-                   "parallelism": "independent server shard per GPU" if world > 1 else "1 GPU"},
-        "bytes_per_step": bytes_, "stage_ms": stage_ms,
-        "pct_of_nominal_8TBs": 100.0 * bytes_["total"] / ms_step / 1e6 / NOMINAL_HBM_GBS,
-        "aggregate_path": {"what": "bookkeeping + masked reduce + bound check only", "GBps": agg_gbs, "ms": agg_ms,
-                           "pct_of_nominal_8TBs": 100.0 * agg_gbs / NOMINAL_HBM_GBS,
-                           "pct_of_%s_peak" % peak_kind: 100.0 * agg_gbs / peak},
-        "roofline": {"kernel": "k_reduce_rows" if work.W <= 4 and work.payload_bytes >= 2048 else "k_reduce_tiled", "bound": "hbm", "achieved": red_gbs, "peak": peak, "peak_kind": peak_kind,
-                     "unit": "GB/s", "frac": red_gbs / peak, "traffic": TRAFFIC.get(work.name),
-                     "algorithmic_bytes_per_launch": bytes_["reduce"], "ms_per_launch": stage_ms["reduce"]},
-        "clocks": clocks, "gpu_launches": launches, "e2e": e2e, "cpu_baseline": cpu, "round_loop": round_loop, "reduce_extras": extras,
+    ring, keys, agg = buf["payload_ring"], buf["slot_key"], buf["agg"]
+    extras = {
+        "reduce_ms": timed(lambda: dblp.dblp_aggregate_reduce(plan, ring, keys, agg, dblp.DBLP_MEAN)),
+        "reduce_norm_ms": timed(lambda: dblp.dblp_aggregate_reduce_ex(plan, ring, keys, agg, dblp.DBLP_MEAN, scratch, norm_out)),
+        "reduce_norm_update_ms": timed(lambda: dblp.dblp_aggregate_reduce_ex(plan, ring, keys, agg, dblp.DBLP_MEAN, scratch,
+                                                                             norm_out, params, 0.01)),
+        "reduce_atomic_order_free_ms": timed(lambda: dblp.dblp_aggregate_reduce_atomic(plan, ring, keys, agg, dblp.DBLP_MEAN)),
+        "grad_norm": float(norm_out[1].item()),
     }
-    print(json.dumps(out))
+    return round_loop, extras
+
+
+def run_gpu(args):
+    job = Job()
+    job.args = args
+    names = [args.workload] if args.workload else [HEADLINE] + list(PER_CONFIG)
+    out = None
+    for i, name in enumerate(names):
+        steps = args.steps if args.steps is not None else DEFAULT_STEPS[name]
+        warmup = max(3, 5 if args.warmup is None else args.warmup)
+        rec, work, bytes_all = measure(job, name, steps, warmup, full=(i == 0))
+        if i == 0:
+            out = rec
+            if job.rank == 0 and job.world == 1 and not args.no_cpu_baseline:
+                out["cpu_baseline"] = cpu_baseline(work)
+            if len(names) > 1:
+                out["per_config"] = []
+        else:
+            keep = ("value", "unit", "ms_per_step", "steps", "warmup", "dtype", "config", "pct_of_nominal_8TBs", "step_GBps",
+                    "bytes_per_step", "stage_ms", "aggregate_path", "roofline", "clocks", "gpu_launches", "verified")
+            out["per_config"].append({k: rec[k] for k in keep} | {k: v for k, v in rec.items() if k.startswith("pct_of_")})
+    if job.dist is not None:
+        job.barrier()
+        job.dist.destroy_process_group()
+    if job.rank == 0:
+        print(json.dumps(out))
 
 
 def run_sweep(args):
     """Stand-alone timing of packetize and of the aggregate path (bookkeeping + reduce + bound check) over the size
-    sweep: per-worker buffer 1 MiB * 4^k, W in {2, 8, 32}, payload {1024, 4096}, 5 % bursty loss.  Points that do not
-    fit in device memory are left out.  Prints one JSON line."""
+    sweep: per-worker buffer 1 MiB * 4^k, W in {1, 2, 8, 32}, payload {1024, 4096}, fp32 and bf16, 5 % bursty loss.
+    Points that do not fit in device memory are left out.  Prints one JSON line."""
     from paper_2605_01989_b200 import binding as dblp
     torch.cuda.set_device(0)
     dev = "cuda:0"
     peak, peak_kind = measured_peak()
     rows = []
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    for k in range(6):
-        for W in (2, 8, 32):
-            for P in (1024, 4096):
-                work = wl.sweep_point((1 << 20) * 4 ** k, W, P, 0.05, "ge", 10)
-                free, _ = torch.cuda.mem_get_info()
-                if work.device_bytes() + (2 << 30) > free:
-                    rows.append({"buffer_MiB": 4 ** k, "W": W, "P": P, "skipped": "does not fit"})
-                    continue
-                plan = dblp.Plan(work.numel, work.dtype, work.payload_bytes, work.W)
-                buf = plan.alloc_round(dev)
-                grads = wl.make_grads(work, dev)
-                model = dblp.loss_model(work.loss.kind, **work.loss.thresholds(plan.C))
-                reps = max(3, min(50, int(2e10 / work.device_bytes())))
+    for dtype in ("f32", "bf16"):
+        for k in range(6):
+            for W in (1, 2, 8, 32):
+                for P in (1024, 4096):
+                    if dtype == "bf16" and k % 2 == 0:
+                        continue                          # bf16: every other size
+                    work = wl.sweep_point((1 << 20) * 4 ** k, W, P, 0.05, "ge", 10)
+                    if dtype == "bf16":                   # same bytes per worker, twice the elements
+                        work.dtype = "bf16"
+                        work.numel = [2 * work.numel[0]]
+                    free, _ = torch.cuda.mem_get_info()
+                    if work.device_bytes() + (2 << 30) > free:
+                        rows.append({"dtype": dtype, "buffer_MiB": 4 ** k, "W": W, "P": P, "skipped": "does not fit"})
+                        continue
+                    plan = dblp.Plan(work.numel, work.dtype, work.payload_bytes, work.W)
+                    buf = plan.alloc_round(dev)
+                    grads = wl.make_grads(work, dev)
+                    model = dblp.loss_model(work.loss.kind, **work.loss.thresholds(plan.C))
+                    reps = max(3, min(50, int(2e10 / work.device_bytes())))
 
-                def timed(fn):
-                    for _ in range(2):
-                        fn()
-                    a.record()
-                    for _ in range(reps):
-                        fn()
-                    b.record()
-                    torch.cuda.synchronize()
-                    return a.elapsed_time(b) / reps
+                    def timed(fn):
+                        for _ in range(2):
+                            fn()
+                        a.record()
+                        for _ in range(reps):
+                            fn()
+                        b.record()
+                        torch.cuda.synchronize()
+                        return a.elapsed_time(b) / reps
 
-                t_pack = timed(lambda: dblp.dblp_packetize(plan, grads, 1, buf["hdr_ring"], buf["payload_ring"]))
-                dblp.dblp_apply_loss(plan, model, work.seed, 1, 0, buf["delivered_bits"], buf["arrival"],
-                                     buf["n_arrived"], buf["ws"])
-
-                def agg_path():
-                    dblp.dblp_round_reset(plan, buf["recv_bitmap"], buf["slot_key"], buf["counters"])
-                    dblp.dblp_aggregate(plan, buf["hdr_ring"], buf["payload_ring"], plan.M, buf["arrival"],
-                                        buf["n_arrived"], plan.M, 1, buf["recv_bitmap"], buf["slot_key"],
-                                        buf["counters"], buf["agg"], dblp.DBLP_MEAN)
-                    dblp.dblp_check_bound(plan, buf["recv_bitmap"], 50000, buf["recv_cnt"], buf["missing_cnt"],
-                                          buf["ok"], buf["all_ok"])
-
-                t_agg = timed(agg_path)
-                t_red = timed(lambda: dblp.dblp_aggregate_reduce(plan, buf["payload_ring"], buf["slot_key"], buf["agg"],
-                                                                 dblp.DBLP_MEAN))
-                n = int(buf["n_arrived"].item())
-                by = byte_model(work, plan.C, n, int(n / plan.M * work.W * work.N * work.elem_size))
-                rows.append({"buffer_MiB": 4 ** k, "W": W, "P": P, "packets": plan.M, "loss": 1 - n / plan.M,
-                             "packetize_GBps": by["packetize"] / t_pack / 1e6,
-                             "aggregate_path_GBps": (by["book"] + by["reduce"] + by["check_bound"]) / t_agg / 1e6,
-                             "reduce_GBps": by["reduce"] / t_red / 1e6, "reduce_frac_of_%s" % peak_kind: by["reduce"] / t_red / 1e6 / peak,
-                             "aggregate_path_us": t_agg * 1e3})
-                plan.close()
-                del buf, grads
-                torch.cuda.empty_cache()
+                    t_pack = timed(lambda: dblp.dblp_packetize(plan, grads, 1, buf["hdr_ring"], buf["payload_ring"]))
+                    dblp.dblp_round_send(plan, grads, model, work.seed, 1, buf)
+                    t_agg = timed(lambda: (dblp.dblp_round_reset(plan, buf["recv_bitmap"], buf["slot_key"], buf["counters"]),
+                                           dblp.dblp_round_receive(plan, 1, 50000, dblp.DBLP_MEAN, buf)))
+                    t_red = timed(lambda: dblp.dblp_aggregate_reduce(plan, buf["payload_ring"], buf["slot_key"], buf["agg"],
+                                                                     dblp.DBLP_MEAN))
+                    n = int(buf["n_arrived"].item())
+                    by = byte_model(work.W, work.N, work.elem_size, plan.C, n, int(n / plan.M * work.W * work.N * work.elem_size))
+                    rows.append({"dtype": dtype, "buffer_MiB": 4 ** k, "W": W, "P": P, "packets": plan.M, "loss": 1 - n / plan.M,
+                                 "kernel": reduce_kernel_name(work),
+                                 "packetize_GBps": by["packetize"] / t_pack / 1e6,
+                                 "aggregate_path_GBps": by["aggregate_path"] / t_agg / 1e6,
+                                 "reduce_GBps": by["reduce"] / t_red / 1e6,
+                                 "reduce_frac_of_%s" % peak_kind: by["reduce"] / t_red / 1e6 / peak,
+                                 "aggregate_path_us": t_agg * 1e3})
+                    plan.close()
+                    del buf, grads
+                    torch.cuda.empty_cache()
     print(json.dumps({"sweep": rows, "peak": peak, "peak_kind": peak_kind}))
 
 
-# DRAM bytes (read + write) per k_reduce launch from an ncu capture of this same workload; None until captured, and
-# reset to None whenever the kernel changes.
-TRAFFIC = {"resnet50-f32": 883.6e6}
-
-
 # ----------------------------------------------------------------------------------------------------------------------
-def oracle_round(op, om, grads, work, rnd):
-    from oracle import dblp_oracle as orc  # noqa: F401
+def oracle_round(op, om, grads, work, rnd, bound):
+    """One whole round by the CPU checker; returns (arrivals, seconds of the whole round, seconds of its aggregate path:
+    bookkeeping + reduce + tolerance test)."""
+    t0 = time.perf_counter()
     hdr, pay = op.packetize(grads, rnd)
     d, _ = op.loss_mask(om, work.seed, rnd)
     arr, n = op.arrival(d, work.seed, rnd)
+    t1 = time.perf_counter()
     st = op.book(hdr, arr, n, rnd, op.new_state())
-    agg = op.reduce(pay, st, mean=True)
-    res = op.check_bound(st["bitmap"], work.bounds_ppm[0])
-    return n, agg, res
+    op.reduce(pay, st, mean=True)
+    op.check_bound(st["bitmap"], bound)
+    t2 = time.perf_counter()
+    return n, t2 - t0, t2 - t1
 
 
-def oracle_setup(work):
+def oracle_setup(work, threads):
     from oracle import dblp_oracle as orc
     op = orc.Plan(work.numel, work.elem_size, work.payload_bytes, work.W)
     om = orc.loss_model(work.loss.kind, **work.loss.thresholds(op.C))
@@ -490,8 +559,7 @@ def oracle_setup(work):
         grads = [g.view(torch.int16).numpy().view("uint16") for g in grads]
     else:
         grads = [g.numpy() for g in grads]
-    threads = orc.set_threads(os.cpu_count() or 1)
-    return op, om, grads, threads
+    return op, om, grads, orc.set_threads(threads)
 
 
 def sample_of(work, max_elems):
@@ -504,54 +572,70 @@ def sample_of(work, max_elems):
             break
         numel.append(min(n, max_elems))
         tot += numel[-1]
-    import copy
     s = copy.copy(work)
     s.numel = numel
     return s, "leading %d of %d tensors (%d of %d elements per worker)" % (len(numel), len(work.numel), tot, work.N)
 
 
-def cpu_baseline(work, gpu_total_bytes):
-    """The CPU checker, as it stands, on a bounded sample of the same workload (about 10-30 s of CPU work)."""
-    sample, what = sample_of(work, 32_000_000)
-    op, om, grads, threads = oracle_setup(sample)
-    oracle_round(op, om, grads, sample, 1)                       # first call pays for page faults of fresh buffers
+def time_oracle(work, sample, what, threads, budget_s, max_reps):
+    from oracle import dblp_oracle as orc
+    op, om, grads, used = oracle_setup(sample, threads)
+    bound = work.bounds_ppm[0]
+    oracle_round(op, om, grads, sample, 1, bound)                   # first call pays for page faults of fresh buffers
     t0 = time.perf_counter()
-    reps = 0
-    while reps < 3 or (time.perf_counter() - t0 < 10.0 and reps < 20):
-        n, _, _ = oracle_round(op, om, grads, sample, 2 + reps)
-        reps += 1
-    dt = (time.perf_counter() - t0) / reps
-    bits_recv = n / op.M
-    b = byte_model(sample, op.C, n, int(bits_recv * sample.W * sample.N * sample.elem_size))
-    return {"value": b["total"] / dt / 1e9, "unit": "GB/s", "cores": threads, "kind": "oracle",
-            "sample": "%s, %d rounds, %.2f s per round; only the reduce loop is multi-threaded" % (what, reps, dt)}
+    reps, t_round, t_agg = 0, 0.0, 0.0
+    while reps < 2 or (time.perf_counter() - t0 < budget_s and reps < max_reps):
+        n, a, b = oracle_round(op, om, grads, sample, 2 + reps, bound)
+        t_round, t_agg, reps = t_round + a, t_agg + b, reps + 1
+    t_round, t_agg = t_round / reps, t_agg / reps
+    by = byte_model(sample.W, sample.N, sample.elem_size, op.C, n, int(n / op.M * sample.W * sample.N * sample.elem_size))
+    orc.set_threads(os.cpu_count() or 1)
+    return {"value": by["aggregate_path"] / t_agg / 1e9, "unit": "GB/s", "cores": used, "kind": "oracle",
+            "sample": "%s, %d rounds, %.2f s per round of which %.2f s in bookkeeping + reduce + tolerance test; only the "
+                      "reduce loop is multi-threaded" % (what, reps, t_round, t_agg),
+            "step_GBps": by["total"] / t_round / 1e9, "ms_per_step": t_round * 1e3}
+
+
+def cpu_baseline(work):
+    """The CPU checker, as it stands, on a bounded sample of the same workload: on all host cores and on one."""
+    sample, what = sample_of(work, 32_000_000)
+    allc = time_oracle(work, sample, what, os.cpu_count() or 1, 10.0, 12)
+    one = time_oracle(work, sample, what, 1, 8.0, 6)
+    allc["single_thread"] = {k: one[k] for k in ("value", "unit", "cores", "sample", "step_GBps")}
+    return allc
 
 
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    work = wl.config(WORKLOADS[args.workload])
+    name = args.workload or HEADLINE
+    work = wl.config(WORKLOADS[name])
     total_steps = args.steps + args.warmup
     budget_s = 150.0
     # about 65 ns per element-worker on one core for packetize + reduce: size the sample so the run fits the budget
     per_step = budget_s / max(1, total_steps)
     max_elems = int(max(1_000_000, min(work.N, per_step / (8e-9 * work.W))))
     sample, what = sample_of(work, max_elems)
-    op, om, grads, threads = oracle_setup(sample)
+    op, om, grads, threads = oracle_setup(sample, os.cpu_count() or 1)
+    bound = work.bounds_ppm[0]
     for i in range(args.warmup):
-        oracle_round(op, om, grads, sample, 1 + i)
-    t0 = time.perf_counter()
+        oracle_round(op, om, grads, sample, 1 + i, bound)
+    t_round = t_agg = 0.0
     for k in range(args.steps):
-        n, _, _ = oracle_round(op, om, grads, sample, 100 + k)
-    dt = (time.perf_counter() - t0) / args.steps
-    b = byte_model(sample, op.C, n, int(n / op.M * sample.W * sample.N * sample.elem_size))
-    v = b["total"] / dt / 1e9
+        n, a, b = oracle_round(op, om, grads, sample, 100 + k, bound)
+        t_round, t_agg = t_round + a, t_agg + b
+    t_round, t_agg = t_round / args.steps, t_agg / args.steps
+    by = byte_model(sample.W, sample.N, sample.elem_size, op.C, n, int(n / op.M * sample.W * sample.N * sample.elem_size))
+    v = by["aggregate_path"] / t_agg / 1e9
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": v, "unit": "GB/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_round * 1e3, "higher_is_better": True,
         "vs_baseline": None, "dtype": work.dtype, "data": "synthetic",
-        "config": {"workload": work.name, "W": work.W, "payload_bytes": work.payload_bytes, "loss": work.loss.kind},
+        "config": {"workload": work.name, "W": work.W, "payload_bytes": work.payload_bytes, "tensors": len(work.numel),
+                   "elements_per_worker": work.N, "loss": work.loss.kind},
+        "value_is": "aggregate path (bookkeeping + masked reduce + tolerance test): its bytes / its time inside the step",
+        "step_GBps": by["total"] / t_round / 1e9,
         "cpu_baseline": {"value": v, "unit": "GB/s", "kind": "oracle", "cores": threads,
                          "sample": what + "; only the reduce loop is multi-threaded"},
         "e2e": {"value": v, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
@@ -562,26 +646,24 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
-    ap.add_argument("--workload", choices=sorted(WORKLOADS), default="resnet50")
+    ap.add_argument("--workload", choices=sorted(WORKLOADS), default=None,
+                    help="one workload only; default: gpt2xl as the headline with resnet50 and bert under per_config")
     ap.add_argument("--impl", choices=["dblp", "reference"], default="dblp")
-    ap.add_argument("--e2e-steps", type=int, default=30)
+    ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-round-loop", action="store_true")
-    ap.add_argument("--serial", action="store_true", help="all stages on one stream")
-    ap.add_argument("--graph", action="store_true", help="replay the step as a CUDA graph (for launch-bound sizes)")
+    ap.add_argument("--no-verify", action="store_true", help="skip the check of the last round against the CPU checker")
+    ap.add_argument("--extras", action="store_true", help="also run the control-loop and fused-reduce side sections")
     ap.add_argument("--sweep", action="store_true", help="time the size sweep instead of the default step")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
         return
     if args.impl == "reference":
-        args.steps = 5 if args.steps is None else args.steps
+        args.steps = 3 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup
         run_reference(args)
     else:
-        args.steps = 1000 if args.steps is None else args.steps
-        args.warmup = max(3, 10 if args.warmup is None else args.warmup)
         run_gpu(args)
 
 

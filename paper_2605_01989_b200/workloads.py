@@ -176,15 +176,32 @@ def sweep(max_device_bytes: Optional[int] = None) -> List[Workload]:
     return pts
 
 
-def make_grads(wl: Workload, device="cpu", workers=None) -> List[torch.Tensor]:
-    """Worker w's flat gradient: N values N(0, sigma^2) from generator seed*1000 + w, cast to the workload's dtype."""
-    out = []
-    for w in (range(wl.W) if workers is None else workers):
+def make_grads(wl: Workload, device="cpu", workers=None, elem_range: Optional[Tuple[int, int]] = None,
+               out: Optional[torch.Tensor] = None) -> List[torch.Tensor]:
+    """Worker w's flat gradient: N values N(0, sigma^2) from generator seed*1000 + w, cast to the workload's dtype.
+    elem_range = (first, last): only that range of each worker's vector is kept (the whole vector is still drawn, so
+    the values are those of the unsplit workload).  out: one tensor of len(workers) * (kept length) elements of the
+    workload's dtype that receives the gradients back to back; the returned list then holds views into it."""
+    ws = list(range(wl.W) if workers is None else workers)
+    lo, hi = (0, wl.N) if elem_range is None else elem_range
+    n = hi - lo
+    res = []
+    for k, w in enumerate(ws):
         g = torch.Generator(device=device)
         g.manual_seed(wl.seed * 1000 + w)
         x = torch.randn(wl.N, generator=g, device=device, dtype=torch.float32)
         x.mul_(wl.sigma)
-        if wl.dtype == "bf16":
-            x = x.to(torch.bfloat16)
-        out.append(x)
-    return out
+        if elem_range is not None:
+            x = x[lo:hi]
+        if out is not None:
+            view = out[k * n:(k + 1) * n]
+            view.copy_(x)                      # casts to bf16 where the workload asks for it
+            res.append(view)
+        else:
+            if wl.dtype == "bf16":
+                x = x.to(torch.bfloat16)
+            elif elem_range is not None:
+                x = x.clone()                  # let go of the whole vector
+            res.append(x)
+        del x
+    return res

@@ -352,6 +352,48 @@ def test_worker_counts_at_the_shared_memory_limit_of_the_tiled_reduce(W, P):
     H.full_round_parity(work([100, 7, 64, 333], "f32", P, W, wl.LossSpec("iid", 0.3), W, bounds=(0, 300000)))
 
 
+@pytest.mark.parametrize("loss", [wl.LossSpec("iid", 0.1), wl.LossSpec("ge", 0.1, 5.0),
+                                  wl.LossSpec("microburst", window_frac=0.2, p_in=0.5, p_out=0.01)], ids=["iid", "ge", "mb"])
+@pytest.mark.parametrize("world", [2, 3, 5])
+def test_shard_plans_side_by_side_equal_the_unsplit_round(loss, world):
+    """A server split over `world` devices, its shards run here one after the other on one device (they do not depend
+    on each other): delivered and received bitmaps side by side, counts summed and aggregates stitched must equal the
+    unsplit round of the oracle -- the loss draws use stream-wide packet numbers."""
+    from paper_2605_01989_b200 import shard
+    numel = [1000, 1, 352 * 40, 353, 7, 100003, 2, 352, 5000, 33]
+    w = work(numel, "f32", 1408, 4, loss, 19, bounds=(50000,))
+    op = orc.Plan(w.numel, 4, 1408, 4)
+    _, om = H.models_for(w, op.C)
+    host = H.to_host(wl.make_grads(w, H.DEV), "f32")        # the runners draw the same values on the device
+    o_hdr, o_pay, o_del, o_arr, o_n, st = H.oracle_round(op, om, host, w.seed, w.round)
+    want_bits = np.unpackbits(st["bitmap"].view(np.uint8).reshape(op.W, -1), axis=1, bitorder="little")[:, :op.C]
+    o_recv, o_miss, o_ok, o_all = op.check_bound(st["bitmap"], 50000)
+
+    specs = shard.shard_specs(w.numel, w.E, world)
+    bits, aggs, recv, miss = [], [], 0, 0
+    for spec in specs:
+        if spec.empty:
+            continue
+        r = shard.GpuShardRunner(w, spec, H.DEV)
+        agg, rc, ms = r.round(w.round, 50000)
+        torch.cuda.synchronize()
+        for name in ("delivered_bits", "recv_bitmap"):               # no junk in this round: the two are equal
+            b = H.u32(r.buf[name]).reshape(op.W, -1)
+            got = np.unpackbits(b.view(np.uint8).reshape(op.W, -1), axis=1, bitorder="little")
+            assert not got[:, spec.chunks:].any(), "padding bits of " + name
+            if name == "recv_bitmap":
+                bits.append(got[:, :spec.chunks])
+        aggs.append(agg.cpu().numpy())
+        recv = recv + H.u32(rc).astype(np.int64)
+        miss = miss + H.u32(ms).astype(np.int64)
+        r.close()
+    H.assert_bits_equal(np.concatenate(bits, axis=1), want_bits, "shards' bitmaps side by side")
+    H.assert_bits_equal(np.concatenate(aggs), op.reduce(o_pay, st, mean=True), "stitched aggregate")
+    assert recv.tolist() == o_recv[:, 0].tolist() and miss.tolist() == o_miss[:, 0].tolist()
+    ok, all_ok = shard.decide(dblp.dblp_bound_ok, torch.from_numpy(recv), torch.from_numpy(miss), 50000)
+    assert ok == o_ok[:, 0].tolist() and all_ok == o_all
+
+
 def test_argument_errors_are_reported_not_faulted():
     w = work(ALIGNED, "f32", 1024, 2, wl.LossSpec("iid", 0.1), 1)
     g = H.GpuRound(w)
