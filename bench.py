@@ -75,6 +75,23 @@ def chunk_lengths(numel, E):
     return np.concatenate([np.minimum(E, n - np.arange(-(-n // E), dtype=np.int64) * E) for n in numel])
 
 
+def workload_by_name(name):
+    """A named workload, or one point of the size sweep written as point:DTYPE:MiB:W:PAYLOAD (for instance
+    point:bf16:64:16:4096 = 16 workers with 64 MiB of bf16 each in 4096-byte packets, 5 % bursty loss, seed 10): the
+    bounded cases that profiler captures run on."""
+    if name.startswith("point:"):
+        _, dtype, mib, W, P = name.split(":")
+        work = wl.sweep_point(int(mib) << 20, int(W), int(P), 0.05, "ge", 10)
+        if dtype == "bf16":                                   # same bytes per worker, twice the elements
+            work.dtype, work.numel = "bf16", [2 * work.numel[0]]
+        elif dtype != "f32":
+            raise SystemExit("point: dtype must be f32 or bf16")
+        work.name = name
+        work.bounds_ppm = (80000,)
+        return work
+    return wl.config(WORKLOADS[name])
+
+
 def reduce_kernel_name(work):
     W, es = work.W, work.elem_size
     if W > 6000:
@@ -186,7 +203,7 @@ def measure(job, name, steps, warmup, full):
     from paper_2605_01989_b200 import binding as dblp
     from paper_2605_01989_b200 import shard
     dev, world, rank = job.dev, job.world, job.rank
-    work = wl.config(WORKLOADS[name])
+    work = workload_by_name(name)
     specs = shard.shard_specs(work.numel, work.E, world)
     spec = specs[rank]
     bound = work.bounds_ppm[-1] if name == "gpt2xl" else work.bounds_ppm[0]
@@ -453,7 +470,7 @@ def run_gpu(args):
     names = [args.workload] if args.workload else [HEADLINE] + list(PER_CONFIG)
     out = None
     for i, name in enumerate(names):
-        steps = args.steps if args.steps is not None else DEFAULT_STEPS[name]
+        steps = args.steps if args.steps is not None else DEFAULT_STEPS.get(name, 50)
         warmup = max(3, 5 if args.warmup is None else args.warmup)
         rec, work, bytes_all = measure(job, name, steps, warmup, full=(i == 0))
         if i == 0:
@@ -610,7 +627,7 @@ def run_reference(args):
     if rank != 0:
         return
     name = args.workload or HEADLINE
-    work = wl.config(WORKLOADS[name])
+    work = workload_by_name(name)
     total_steps = args.steps + args.warmup
     budget_s = 150.0
     # about 65 ns per element-worker on one core for packetize + reduce: size the sample so the run fits the budget
@@ -646,8 +663,9 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
-    ap.add_argument("--workload", choices=sorted(WORKLOADS), default=None,
-                    help="one workload only; default: gpt2xl as the headline with resnet50 and bert under per_config")
+    ap.add_argument("--workload", default=None,
+                    help="one workload only (%s, or point:DTYPE:MiB:W:PAYLOAD for one point of the size sweep); default: "
+                         "gpt2xl as the headline with resnet50 and bert under per_config" % ", ".join(sorted(WORKLOADS)))
     ap.add_argument("--impl", choices=["dblp", "reference"], default="dblp")
     ap.add_argument("--e2e-steps", type=int, default=10)
     ap.add_argument("--no-e2e", action="store_true")
@@ -656,6 +674,8 @@ def main():
     ap.add_argument("--extras", action="store_true", help="also run the control-loop and fused-reduce side sections")
     ap.add_argument("--sweep", action="store_true", help="time the size sweep instead of the default step")
     args = ap.parse_args()
+    if args.workload is not None and args.workload not in WORKLOADS and not args.workload.startswith("point:"):
+        ap.error("unknown workload %r" % args.workload)
     if args.sweep:
         run_sweep(args)
         return

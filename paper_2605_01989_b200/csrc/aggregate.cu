@@ -35,22 +35,13 @@ struct HeaderView {
     uint32_t worker, seq, round;
 };
 
-__device__ __forceinline__ HeaderView validate_header(const dblp_hdr_t* __restrict__ hdr_ring, uint32_t hdr_stride,
-                                                      uint32_t slot, uint64_t n_slots,
-                                                      const uint4* __restrict__ tensor_tab, uint32_t T, uint32_t W,
-                                                      uint32_t E, uint32_t es)
+// The check itself, on a header (h0 = seq, round, len_bytes, tensor_id; h1 = offset low, offset high, worker,
+// reserved) whose worker and tensor are in range and on that tensor's table entry.
+__device__ __forceinline__ bool header_matches_plan(const uint4& h0, const uint4& h1, const uint4& tt, uint32_t E, uint32_t es)
 {
-    HeaderView h{false, 0u, 0u, 0u};
-    if (slot >= n_slots) return h;
-    const uint4* hp = reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(hdr_ring) + (uint64_t)slot * hdr_stride);
-    const uint4 h0 = __ldg(hp);       // seq, round, len_bytes, tensor_id
-    const uint4 h1 = __ldg(hp + 1);   // offset low, offset high, worker, reserved
-    h.worker = h1.z; h.seq = h0.x; h.round = h0.y;
-    if (h1.z >= W || h0.w >= T) return h;
-    const uint4 tt = __ldg(&tensor_tab[h0.w]);
     const uint64_t nt = (uint64_t)tt.x | ((uint64_t)tt.y << 32);
     const uint64_t off = (uint64_t)h1.x | ((uint64_t)h1.y << 32);
-    if (off >= nt) return h;
+    if (off >= nt) return false;
     uint64_t q;
     bool on_boundary;
     if (h1.y == 0) {                  // offsets below 2^32 (all but the largest tensors): 32-bit division
@@ -62,7 +53,41 @@ __device__ __forceinline__ HeaderView validate_header(const dblp_hdr_t* __restri
         on_boundary = q * E == off;
     }
     const uint64_t len = min((uint64_t)E, nt - off);
-    h.valid = on_boundary && (h0.z == len * es) && (h0.x == tt.z + q);
+    return on_boundary && (h0.z == len * es) && (h0.x == tt.z + q);
+}
+
+__device__ __forceinline__ const uint4* header_ptr(const dblp_hdr_t* __restrict__ hdr_ring, uint32_t hdr_stride, uint32_t slot)
+{
+    return reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(hdr_ring) + (uint64_t)slot * hdr_stride);
+}
+
+// Reads a 32-byte header: one 256-bit load where every header of the ring is 32-byte aligned (wide, the same for all
+// threads of a launch), otherwise two 128-bit loads.
+__device__ __forceinline__ void load_header(const uint4* hp, bool wide, uint4& h0, uint4& h1)
+{
+    if (wide) {
+        asm volatile("ld.global.nc.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=r"(h0.x), "=r"(h0.y), "=r"(h0.z), "=r"(h0.w), "=r"(h1.x), "=r"(h1.y), "=r"(h1.z), "=r"(h1.w)
+                     : "l"(hp));
+    } else {
+        h0 = __ldg(hp);
+        h1 = __ldg(hp + 1);
+    }
+}
+
+__device__ __forceinline__ HeaderView validate_header(const dblp_hdr_t* __restrict__ hdr_ring, uint32_t hdr_stride,
+                                                      uint32_t slot, uint64_t n_slots,
+                                                      const uint4* __restrict__ tensor_tab, uint32_t T, uint32_t W,
+                                                      uint32_t E, uint32_t es)
+{
+    HeaderView h{false, 0u, 0u, 0u};
+    if (slot >= n_slots) return h;
+    const uint4* hp = header_ptr(hdr_ring, hdr_stride, slot);
+    const uint4 h0 = __ldg(hp);
+    const uint4 h1 = __ldg(hp + 1);
+    h.worker = h1.z; h.seq = h0.x; h.round = h0.y;
+    if (h1.z >= W || h0.w >= T) return h;
+    h.valid = header_matches_plan(h0, h1, __ldg(&tensor_tab[h0.w]), E, es);
     return h;
 }
 
@@ -83,10 +108,34 @@ __device__ __forceinline__ void block_count3(bool a, bool b, bool c, uint32_t* s
     __syncthreads();
 }
 
-// One thread per arrival entry.  The claim is a 64-bit atomic minimum that nobody waits for (no return value): who
-// won a cell is settled by the minimum itself, and how many cells were newly won is counted afterwards by k_bitmap from
-// the bitmap words it rewrites.  Here every valid packet of this round is provisionally counted as a repeat
-// (n_dup); k_bitmap moves the newly set bits from n_dup to n_accepted.
+// The same for three small per-thread counts: warp sums, one shared-memory atomic per warp and non-zero sum.
+__device__ __forceinline__ void block_sum3(uint32_t a, uint32_t b, uint32_t c, uint32_t* s_cnt)
+{
+    if (threadIdx.x < 3) s_cnt[threadIdx.x] = 0;
+    __syncthreads();
+    const uint32_t na = __reduce_add_sync(0xFFFFFFFFu, a);
+    const uint32_t nb = __reduce_add_sync(0xFFFFFFFFu, b);
+    const uint32_t nc = __reduce_add_sync(0xFFFFFFFFu, c);
+    if ((threadIdx.x & 31) == 0) {
+        if (na) atomicAdd(&s_cnt[0], na);
+        if (nb) atomicAdd(&s_cnt[1], nb);
+        if (nc) atomicAdd(&s_cnt[2], nc);
+    }
+    __syncthreads();
+}
+
+// A thread takes kBookItems arrival entries, a block's worth apart, and goes through them stage by stage -- all arrival
+// entries, then all headers, then all table entries, then the claims -- so that the loads of a stage are in flight
+// together: the kernel is a chain of dependent random accesses and is bound by their latency, not by bytes.
+// The claim is a 64-bit atomic minimum that nobody waits for (no return value): who won a cell is settled by the
+// minimum itself, and how many cells were newly won is counted afterwards by k_bitmap from the bitmap words it
+// rewrites.  Here every valid packet of this round is provisionally counted as a repeat (n_dup); k_bitmap moves the
+// newly set bits from n_dup to n_accepted.
+#ifndef DBLP_BOOK_ITEMS
+#define DBLP_BOOK_ITEMS 2   // measured on B200: 2 is 10 % ahead of 1 at 2.6 M packets, 4 is behind both
+#endif
+constexpr int kBookItems = DBLP_BOOK_ITEMS;
+
 __global__ void __launch_bounds__(kBookThreads)
 k_book(const dblp_hdr_t* __restrict__ hdr_ring, uint64_t n_slots, const uint32_t* __restrict__ arrival,
        const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap, uint32_t round,
@@ -95,22 +144,43 @@ k_book(const dblp_hdr_t* __restrict__ hdr_ring, uint64_t n_slots, const uint32_t
        uint32_t hdr_stride)
 {
     __shared__ uint32_t s_cnt[3];
+    const bool wide = ((reinterpret_cast<uintptr_t>(hdr_ring) | hdr_stride) & 31u) == 0;
     const uint64_t n = min(*n_arrived_dev, arrival_cap);
-    const uint64_t a = (uint64_t)blockIdx.x * kBookThreads + threadIdx.x;
-    if ((uint64_t)blockIdx.x * kBookThreads >= n) return;          // whole block past the end
+    const uint64_t a0 = (uint64_t)blockIdx.x * (kBookThreads * kBookItems) + threadIdx.x;
+    if ((uint64_t)blockIdx.x * (kBookThreads * kBookItems) >= n) return;   // whole block past the end
     const uint64_t first_number = counters->n_arrived;             // arrival numbers continue across calls of a round
-    bool current = false, stale = false, invalid = false;
-    if (a < n) {
-        const uint32_t slot = __ldg(&arrival[a]);
-        const HeaderView h = validate_header(hdr_ring, hdr_stride, slot, n_slots, tensor_tab, T, W, E, es);
-        if (!h.valid) invalid = true;
-        else if (h.round != round) stale = true;
+    uint32_t slot[kBookItems];
+    uint4 h0[kBookItems], h1[kBookItems], tt[kBookItems];
+    uint32_t live = 0, n_current = 0, n_stale = 0, n_invalid = 0;  // live bit k: item k is still a candidate
+#pragma unroll
+    for (int k = 0; k < kBookItems; ++k) {
+        const uint64_t a = a0 + (uint64_t)k * kBookThreads;
+        if (a < n) { slot[k] = __ldg(&arrival[a]); live |= 1u << k; }
+    }
+#pragma unroll
+    for (int k = 0; k < kBookItems; ++k) {
+        if (!((live >> k) & 1u)) continue;
+        if (slot[k] >= n_slots) { live &= ~(1u << k); ++n_invalid; continue; }
+        load_header(header_ptr(hdr_ring, hdr_stride, slot[k]), wide, h0[k], h1[k]);
+    }
+#pragma unroll
+    for (int k = 0; k < kBookItems; ++k) {
+        if (!((live >> k) & 1u)) continue;
+        if (h1[k].z >= W || h0[k].w >= T) { live &= ~(1u << k); ++n_invalid; continue; }
+        tt[k] = __ldg(&tensor_tab[h0[k].w]);
+    }
+#pragma unroll
+    for (int k = 0; k < kBookItems; ++k) {
+        if (!((live >> k) & 1u)) continue;
+        if (!header_matches_plan(h0[k], h1[k], tt[k], E, es)) ++n_invalid;
+        else if (h0[k].y != round) ++n_stale;
         else {
-            current = true;
-            atomicMin(&slot_key[(uint64_t)h.worker * C + h.seq], ((first_number + a) << 32) | slot);
+            ++n_current;
+            const uint64_t a = a0 + (uint64_t)k * kBookThreads;
+            atomicMin(&slot_key[(uint64_t)h1[k].z * C + h0[k].x], ((first_number + a) << 32) | slot[k]);
         }
     }
-    block_count3(current, stale, invalid, s_cnt);
+    block_sum3(n_current, n_stale, n_invalid, s_cnt);
     if (threadIdx.x == 0) {
         if (s_cnt[0]) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_dup), (unsigned long long)s_cnt[0]);
         if (s_cnt[1]) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_stale), (unsigned long long)s_cnt[1]);
@@ -390,7 +460,7 @@ __device__ __forceinline__ void st_agg16(float* p, float a, float b, float c, fl
 
 
 // ------------------------------------------------------------------------------------------------ tiled reduce
-// Persistent blocks walk over tiles of CH consecutive chunks.  For each tile the W x CH slot entries and the CH chunk
+// Persistent blocks walk over tiles of CH consecutive chunks, from the last tile down.  For each tile the W x CH slot entries and the CH chunk
 // descriptors are brought into shared memory with cp.async while the previous tile is still being summed (two
 // buffers), so the only global loads a thread waits for are the payload vectors themselves: WB * J independent
 // 128-bit loads per thread, issued together, then added in worker order.  A thread's J items are 256 vectors apart,
@@ -410,6 +480,11 @@ __device__ __forceinline__ void st_agg16(float* p, float a, float b, float c, fl
 #define DBLP_REDUCE_J_WIDE 1      // items per thread when W > 4 (8 workers per batch)
 #endif
 constexpr int kTileThreads = DBLP_REDUCE_THREADS;
+
+// The tile a block sums in its turn-th step (turn = blockIdx.x, blockIdx.x + gridDim.x, ...): the last tile first.
+// Right after packetize the most recently written ring slots are the ones still in L2, and those are the last tiles';
+// on a ring a few times the L2 this order was worth 2 % of the reduce's time, on large rings it makes no difference.
+__device__ __forceinline__ uint32_t tile_of_turn(uint32_t turn, uint32_t n_tiles) { return n_tiles - 1 - turn; }
 constexpr int kJWide = DBLP_REDUCE_J_WIDE;
 constexpr size_t kNormSmem = (kTileThreads / 32) * sizeof(double);   // static shared memory of the tiled kernels
 
@@ -610,12 +685,12 @@ k_reduce_tiled(const uint8_t* __restrict__ ring, const unsigned long long* __res
     // i / VPC for i < CH * VPC: exact because the plan keeps CH * VPC * VPC <= 2^32
     auto chunk_of = [&](uint32_t i) { return VPC == 1 ? i : __umulhi(i, vpc_magic); };
 
-    uint32_t tile = blockIdx.x, buf = 0;
-    if (tile < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, tile, 0, CH, C, W);
+    uint32_t turn = blockIdx.x, buf = 0;
+    if (turn < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, tile_of_turn(turn, n_tiles), 0, CH, C, W);
     cp_async_commit();
-    for (; tile < n_tiles; tile += gridDim.x, buf ^= 1) {
-        const uint32_t next = tile + gridDim.x;
-        if (next < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, next, buf ^ 1, CH, C, W);
+    for (; turn < n_tiles; turn += gridDim.x, buf ^= 1) {
+        const uint32_t tile = tile_of_turn(turn, n_tiles), next = turn + gridDim.x;
+        if (next < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, tile_of_turn(next, n_tiles), buf ^ 1, CH, C, W);
         cp_async_commit();
         cp_async_wait<1>();                   // everything but the group just committed has landed
         __syncthreads();
@@ -713,12 +788,12 @@ k_reduce_rows(const uint8_t* __restrict__ ring, const unsigned long long* __rest
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint2* cells = reinterpret_cast<const uint2*>(slot_key);
 
-    uint32_t tile = blockIdx.x, buf = 0;
-    if (tile < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, tile, 0, CH, C, W);
+    uint32_t turn = blockIdx.x, buf = 0;
+    if (turn < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, tile_of_turn(turn, n_tiles), 0, CH, C, W);
     cp_async_commit();
-    for (; tile < n_tiles; tile += gridDim.x, buf ^= 1) {
-        const uint32_t next = tile + gridDim.x;
-        if (next < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, next, buf ^ 1, CH, C, W);
+    for (; turn < n_tiles; turn += gridDim.x, buf ^= 1) {
+        const uint32_t tile = tile_of_turn(turn, n_tiles), next = turn + gridDim.x;
+        if (next < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, tile_of_turn(next, n_tiles), buf ^ 1, CH, C, W);
         cp_async_commit();
         cp_async_wait<1>();
         __syncthreads();
@@ -929,7 +1004,7 @@ extern "C" int dblp_aggregate_claim(const dblp_plan_t* plan, const dblp_hdr_t* h
     DBLP_REQUIRE(n_slots < 0xFFFFFFFFull, DBLP_ECAPACITY, "aggregate_claim: ring has too many slots");
     DBLP_REQUIRE(arrival_cap < (1ull << 32), DBLP_ECAPACITY, "aggregate_claim: arrival list too long");
     if (arrival_cap == 0) return DBLP_OK;
-    const unsigned grid = (unsigned)((arrival_cap + kBookThreads - 1) / kBookThreads);
+    const unsigned grid = (unsigned)((arrival_cap + kBookThreads * kBookItems - 1) / (kBookThreads * kBookItems));
     k_book<<<grid, kBookThreads, 0, static_cast<cudaStream_t>(stream)>>>(
         hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, reinterpret_cast<unsigned long long*>(slot_key), counters,
         plan->d_tensor_tab, plan->T, plan->W, plan->C, plan->E, plan->es, plan->hdr_stride);

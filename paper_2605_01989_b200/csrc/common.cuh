@@ -114,6 +114,11 @@ struct dblp_plan {
     // 0 = the simple one-vector-per-thread kernel
     uint32_t red_variant, red_CH, red_tiles, red_grid, red_rows;
     size_t red_smem;
+    // block order of packetize: 1 = tile by tile with all workers of a tile together, 0 = worker by worker.
+    // Tile-major leaves the end of every worker's ring in L2, which is where the masked reduce starts reading (it
+    // walks the tiles from the last one down); it pays while the ring is only a few times the L2 and costs about 2 %
+    // of the copy rate on rings of many GB, so the plan picks it for rings up to 16 times the L2.
+    uint32_t pack_tile_major;
 };
 
 namespace dblp {

@@ -3,8 +3,10 @@
 // A pure copy, bound by HBM.  A block owns a tile of CH consecutive chunks of one worker: it first brings the tile's
 // chunk descriptors into shared memory (so that no payload load waits on a table lookup), writes the tile's headers,
 // then streams the tile's 16-byte vectors, kPackUnroll per thread per pass with all loads issued before the first
-// store.  The source follows the descriptors, so tensors of any size are handled: a vector that is ragged (end of a short chunk) or whose source is not 16-byte
-// aligned is assembled from element loads, and the slot's tail is written as zero.
+// store.  The source follows the descriptors, so tensors of any size are handled: a vector that is ragged (end of a
+// short chunk) or whose source is not 16-byte aligned is assembled from element loads, and the slot's tail is written
+// as zero.  Blocks run either worker by worker (grid.y = worker) or tile by tile with a tile's workers side by side
+// (one-dimensional grid, nw_fast = workers of the launch); the plan chooses, see dblp_plan::pack_tile_major.
 #include "common.cuh"
 
 namespace dblp {
@@ -45,16 +47,21 @@ __device__ __forceinline__ void st_keep16(void* p, uint4 v)
 
 template <int ES>
 __global__ void __launch_bounds__(kPackThreads)
-k_packetize(GradPtrs grads, uint32_t w0, uint32_t C, uint32_t VPC, uint32_t pay_stride, uint32_t hdr_stride, uint32_t CH,
+k_packetize(GradPtrs grads, uint32_t w0, uint32_t nw_fast, uint32_t C, uint32_t VPC, uint32_t pay_stride, uint32_t hdr_stride, uint32_t CH,
             uint32_t round,
             const uint64_t* __restrict__ chunk_desc, const uint32_t* __restrict__ chunk_tensor,
             const uint64_t* __restrict__ tensor_base, dblp_hdr_t* __restrict__ hdr_ring, uint8_t* __restrict__ ring)
 {
     constexpr uint32_t VE = 16 / ES;
     __shared__ uint64_t s_desc[kPackMaxTile];
-    const uint32_t wl = blockIdx.y, w = w0 + wl, tid = threadIdx.x;
+    uint32_t tile = blockIdx.x, wl = blockIdx.y;
+    if (nw_fast) {                                      // tile-major: consecutive blocks are the workers of one tile
+        tile = blockIdx.x / nw_fast;
+        wl = blockIdx.x - tile * nw_fast;
+    }
+    const uint32_t w = w0 + wl, tid = threadIdx.x;
     const uint8_t* __restrict__ g = static_cast<const uint8_t*>(grads.p[wl]);
-    const uint32_t c0 = blockIdx.x * CH, nch = min(CH, C - c0);
+    const uint32_t c0 = tile * CH, nch = min(CH, C - c0);
     const uint64_t slot0 = (uint64_t)w * C + c0;
 
     for (uint32_t k = tid; k < nch; k += kPackThreads) {
@@ -113,17 +120,18 @@ int packetize_workers(const dblp_plan* plan, const void* const* grads, uint32_t 
     uint32_t CH = (4096u + plan->VPC - 1) / plan->VPC;          // about 64 KB of payload per block
     if (CH > kPackMaxTile) CH = kPackMaxTile;
     const uint64_t gx = (plan->C + CH - 1) / CH;
-    DBLP_REQUIRE(gx < (1ull << 31), DBLP_ECAPACITY, "packetize: grid too large");
+    DBLP_REQUIRE(gx * kMaxWorkersPerLaunch < (1ull << 31), DBLP_ECAPACITY, "packetize: grid too large");
     for (uint32_t w0 = w_first; w0 < w_first + n_workers; w0 += kMaxWorkersPerLaunch) {
         const uint32_t nw = min(kMaxWorkersPerLaunch, w_first + n_workers - w0);
         GradPtrs gp{};
         for (uint32_t k = 0; k < nw; ++k) gp.p[k] = grads[w0 - w_first + k];
-        dim3 grid((unsigned)gx, nw);
+        const uint32_t nw_fast = plan->pack_tile_major ? nw : 0u;
+        const dim3 grid = nw_fast ? dim3((unsigned)(gx * nw), 1) : dim3((unsigned)gx, nw);
         if (plan->es == 4)
-            k_packetize<4><<<grid, kPackThreads, 0, s>>>(gp, w0, (uint32_t)plan->C, plan->VPC, plan->pay_stride, plan->hdr_stride, CH, round,
+            k_packetize<4><<<grid, kPackThreads, 0, s>>>(gp, w0, nw_fast, (uint32_t)plan->C, plan->VPC, plan->pay_stride, plan->hdr_stride, CH, round,
                 plan->d_chunk_desc, plan->d_chunk_tensor, plan->d_base, hdr_ring, static_cast<uint8_t*>(payload_ring) + plan->pay_off);
         else
-            k_packetize<2><<<grid, kPackThreads, 0, s>>>(gp, w0, (uint32_t)plan->C, plan->VPC, plan->pay_stride, plan->hdr_stride, CH, round,
+            k_packetize<2><<<grid, kPackThreads, 0, s>>>(gp, w0, nw_fast, (uint32_t)plan->C, plan->VPC, plan->pay_stride, plan->hdr_stride, CH, round,
                 plan->d_chunk_desc, plan->d_chunk_tensor, plan->d_base, hdr_ring, static_cast<uint8_t*>(payload_ring) + plan->pay_off);
         DBLP_LAUNCHED();
     }

@@ -145,6 +145,10 @@ static int plan_create(const uint64_t* tensor_numel, uint32_t T, int dtype, uint
     DBLP_REQUIRE(e == cudaSuccess, DBLP_ECUDA, "plan: device table setup failed: %s", cudaGetErrorString(e));
     const int rc = configure_reduce(p, 0, 0);
     if (rc != DBLP_OK) return rc;
+    int l2_bytes = 0;
+    e = cudaDeviceGetAttribute(&l2_bytes, cudaDevAttrL2CacheSize, p->device);
+    DBLP_REQUIRE(e == cudaSuccess, DBLP_ECUDA, "plan: device query failed: %s", cudaGetErrorString(e));
+    p->pack_tile_major = p->M * (uint64_t)payload_bytes <= 16ull * (uint64_t)l2_bytes ? 1u : 0u;
     guard.p = nullptr;
     *out = p;
     return DBLP_OK;
