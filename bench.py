@@ -42,10 +42,21 @@ DEFAULT_STEPS = {"flat": 2000, "resnet50": 500, "bert": 100, "gpt2xl": 40, "swee
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes (read + write) that ncu counted for one launch of the reduce kernel, as a ratio to the launch's
-# algorithmic bytes, from a capture of a sweep point of about 1 GB (the bench workloads are too large to capture);
-# `traffic` scales it to the launch that is timed here.  An entry is removed whenever its kernel changes.
-NCU_TRAFFIC = {}
+# DRAM bytes (read + write) that ncu counted for one launch of the reduce kernel, as a ratio to that launch's
+# algorithmic bytes.  The ResNet-50-shaped workload was captured itself; the two large ones are too big to capture, so
+# their ratio comes from a point of the size sweep that runs the same kernel with the same payload size on about 2 GB,
+# and `traffic` scales it to the launch timed here (traffic grows in proportion to the bytes moved).  `commit` is the
+# revision of the kernels the counters were taken on: an entry is removed whenever its kernel changes.
+NCU_TRAFFIC = {
+    "resnet50-f32": {"kernel": "k_reduce_tiled<4, 8, 1, false>", "dram_bytes_per_algorithmic_byte": 0.969,
+                     "captured_on": "resnet50-f32", "commit": "5ca6832", "source": "profiles/k_reduce_tiled_resnet50.md"},
+    "bert-large-bf16": {"kernel": "k_reduce_tiled<2, 8, 1, false>", "dram_bytes_per_algorithmic_byte": 0.975,
+                        "captured_on": "point:bf16:64:16:4096", "commit": "5ca6832",
+                        "source": "profiles/k_reduce_tiled_sweep_points_bf16_f32.md"},
+    "gpt2-xl-f32": {"kernel": "k_reduce_tiled<4, 8, 1, false>", "dram_bytes_per_algorithmic_byte": 0.978,
+                    "captured_on": "point:f32:128:8:4096", "commit": "5ca6832",
+                    "source": "profiles/k_reduce_tiled_sweep_points_bf16_f32.md"},
+}
 
 
 def measured_peak():
@@ -281,7 +292,9 @@ def measure(job, name, steps, warmup, full):
     red_gbs = mine["reduce"] / stage_ms["reduce"] / 1e6 if stage_ms["reduce"] else 0.0
     agg_gbs = bytes_all["aggregate_path"] / agg_ms / 1e6
     kernel = reduce_kernel_name(work)
-    ncu = NCU_TRAFFIC.get(kernel)
+    ncu = NCU_TRAFFIC.get(work.name) if world == 1 else None
+    if ncu is not None and ncu["kernel"] != kernel:
+        ncu = None
     rec = {
         "metric": METRIC, "value": agg_gbs, "unit": "GB/s", "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "vs_baseline": None, "dtype": work.dtype, "data": "synthetic",
@@ -305,7 +318,8 @@ def measure(job, name, steps, warmup, full):
         "roofline": {"kernel": kernel, "bound": "hbm", "achieved": red_gbs, "peak": peak, "peak_kind": peak_kind,
                      "unit": "GB/s", "frac": red_gbs / peak,
                      "traffic": ncu["dram_bytes_per_algorithmic_byte"] * mine["reduce"] if ncu else None,
-                     "traffic_source": ncu["source"] if ncu else None,
+                     "traffic_source": {k: ncu[k] for k in ("source", "captured_on", "commit", "dram_bytes_per_algorithmic_byte")}
+                     if ncu else None,
                      "algorithmic_bytes_per_launch": mine["reduce"], "ms_per_launch": stage_ms["reduce"]},
         "clocks": clocks, "gpu_launches": launches, "verified": verified,
     }
