@@ -458,6 +458,14 @@ __device__ __forceinline__ void st_agg16(float* p, float a, float b, float c, fl
     asm volatile("st.global.cs.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 
+// Eight fp32 results of a bf16 vector as one 256-bit store: the lane's whole 32-byte sector in one request (two 128-bit
+// stores at a 32-byte stride would each fill half of every sector they touch).  p must be 32-byte aligned.
+__device__ __forceinline__ void st_agg32(float* p, const float (&a)[8])
+{
+    asm volatile("st.global.cs.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(a[0]), "f"(a[1]), "f"(a[2]), "f"(a[3]),
+                 "f"(a[4]), "f"(a[5]), "f"(a[6]), "f"(a[7])
+                 : "memory");
+}
 
 // ------------------------------------------------------------------------------------------------ tiled reduce
 // Persistent blocks walk over tiles of CH consecutive chunks, from the last tile down.  For each tile the W x CH slot entries and the CH chunk
@@ -571,8 +579,15 @@ __device__ __forceinline__ void finish_vector(float (&acc)[16 / ES], float* __re
                 if (e < (int)nv) out16[e] = (uint16_t)bf16_rne(acc[e]);
         }
     } else if (nv == VE && (reinterpret_cast<uintptr_t>(out) & 15u) == 0) {
-#pragma unroll
-        for (int q = 0; q < VE / 4; ++q) st_agg16(out + 4 * q, acc[4 * q], acc[4 * q + 1], acc[4 * q + 2], acc[4 * q + 3]);
+        if constexpr (VE == 8) {
+            if ((reinterpret_cast<uintptr_t>(out) & 31u) == 0) st_agg32(out, acc);
+            else {
+                st_agg16(out, acc[0], acc[1], acc[2], acc[3]);
+                st_agg16(out + 4, acc[4], acc[5], acc[6], acc[7]);
+            }
+        } else {
+            st_agg16(out, acc[0], acc[1], acc[2], acc[3]);
+        }
     } else {
 #pragma unroll
         for (int e = 0; e < VE; ++e)
