@@ -392,8 +392,15 @@ def end_to_end(job, work, runner, bound, mine, steps):
         agg_host = torch.empty(n_local, dtype=torch.float32, pin_memory=True)
     except RuntimeError:
         pinned = False
-        grads_host = [torch.empty(n_local, dtype=dtype) for _ in range(work.W)]
-        agg_host = torch.empty(n_local, dtype=torch.float32)
+        grads_host = agg_host = None
+        try:
+            grads_host = [torch.empty(n_local, dtype=dtype) for _ in range(work.W)]
+            agg_host = torch.empty(n_local, dtype=torch.float32)
+        except (RuntimeError, MemoryError) as e:       # the host cannot hold a copy of the gradients at all
+            del grads_host, agg_host
+            return {"value": None, "unit": "GB/s", "h2d_bytes_per_step": None, "d2h_bytes_per_step": None,
+                    "unavailable": "host memory for %d x %d bytes of gradients: %s" % (work.W, n_local * work.elem_size,
+                                                                                       str(e)[:160])}
     for h, g in zip(grads_host, runner.grads):
         h.copy_(g)
     grads_dev = runner.grads_dev                  # the workers' gradients back to back: the copies land where they already are
@@ -482,6 +489,15 @@ def run_gpu(args):
     job = Job()
     job.args = args
     names = [args.workload] if args.workload else [HEADLINE] + list(PER_CONFIG)
+    left_out = []
+    if not args.workload:
+        # the headline is the largest workload that fits in what is free on this device (a rank holds 1 / world of it)
+        free, _ = torch.cuda.mem_get_info()
+        need = lambda n: workload_by_name(n).device_bytes() // job.world + (4 << 30)                     # noqa: E731
+        left_out = [n for n in names if need(n) > free]
+        names = sorted([n for n in names if n not in left_out], key=need, reverse=True)
+        if not names:
+            raise SystemExit("bench.py: no workload fits in %.1f GB of free device memory" % (free / 1e9))
     out = None
     for i, name in enumerate(names):
         steps = args.steps if args.steps is not None else DEFAULT_STEPS.get(name, 50)
@@ -497,6 +513,8 @@ def run_gpu(args):
             keep = ("value", "unit", "ms_per_step", "steps", "warmup", "dtype", "config", "pct_of_nominal_8TBs", "step_GBps",
                     "bytes_per_step", "stage_ms", "aggregate_path", "roofline", "clocks", "gpu_launches", "verified")
             out["per_config"].append({k: rec[k] for k in keep} | {k: v for k, v in rec.items() if k.startswith("pct_of_")})
+    if left_out:
+        out["config"]["left_out"] = "%s: not enough free device memory" % ", ".join(left_out)
     if job.dist is not None:
         job.barrier()
         job.dist.destroy_process_group()
