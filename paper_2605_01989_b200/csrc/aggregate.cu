@@ -2,13 +2,15 @@
 // (Algorithm 2: integrity check, bitmap update, zero fill, reconstruction; Algorithm 3: mean over all workers;
 // Section III-A: packets of another round are dropped).
 //
-// k_book    one thread per arrival entry: 32-byte header read, checks against the plan's tables, one 64-bit atomic
+// k_book    two arrival entries per thread: 32-byte header read, checks against the plan's tables, one 64-bit atomic
 //           minimum on the claimed cell.  Integer atomics only, so every result is independent of thread order.
-// k_bitmap  warp ballot over the cells of a row -> one bitmap word per warp; also folds this call's arrival count
-//           into the counters (after every k_book thread has read the old value).
+// k_bitmap  warp ballot over the cells of a row -> one bitmap word per warp; counts the newly set bits (the packets
+//           this call accepted) and folds this call's arrival count into the counters (after every k_book thread
+//           has read the old value).
 // k_reduce_tiled  the bandwidth-bound kernel: one thread per (chunk, 16-byte vector), tables of a tile of chunks
 //           staged in shared memory, eight 128-bit streaming payload loads in flight per thread, fp32 additions in
-//           worker order, 128-bit streaming stores.  A worker whose packet was lost costs no payload traffic.
+//           worker order, streaming stores of 128 bits (fp32 input) or 256 bits (bf16 input: eight results per
+//           vector).  A worker whose packet was lost costs no payload traffic.
 // k_reduce_rows   the same with a warp per chunk; chosen for few workers with long payloads.
 // k_reduce  the simple form (tables read from global memory), kept for worker counts whose slot entries do not
 //           fit in shared memory.
