@@ -119,6 +119,9 @@ struct dblp_plan {
     // walks the tiles from the last one down); it pays while the ring is only a few times the L2 and costs about 2 %
     // of the copy rate on rings of many GB, so the plan picks it for rings up to 16 times the L2.
     uint32_t pack_tile_major;
+    // dblp_round_reset as one kernel that leaves the claim table in L2 (tables up to a quarter of the L2), instead of
+    // three memsets
+    uint32_t reset_in_l2;
 };
 
 namespace dblp {

@@ -45,7 +45,7 @@ def test_record_of_a_small_workload_has_the_contract_keys_and_is_verified():
     assert "scaling" not in rec                                   # one GPU: nothing scales
     assert rec["config"]["workload"] == work.name == "flat-1M-f32" and rec["dtype"] == "f32" and rec["vs_baseline"] is None
     assert rec["verified"]["ok"] and all(rec["verified"]["checks"].values())
-    assert rec["gpu_launches"] == 5 * 9                           # pointwise loss model: nine kernels per round
+    assert rec["gpu_launches"] == 5 * 10                          # pointwise loss model: ten kernels per round (one of them the round reset)
     roof = rec["roofline"]
     assert roof["bound"] == "hbm" and roof["unit"] == "GB/s" and roof["achieved"] > 0
     assert abs(roof["frac"] - roof["achieved"] / roof["peak"]) < 1e-12
