@@ -498,21 +498,22 @@ def run_gpu(args):
         names = sorted([n for n in names if n not in left_out], key=need, reverse=True)
         if not names:
             raise SystemExit("bench.py: no workload fits in %.1f GB of free device memory" % (free / 1e9))
-    out = None
-    for i, name in enumerate(names):
+    # the smaller workloads run first, on a device that has held nothing large yet; names[0] is the headline
+    out, others = None, []
+    keep = ("value", "unit", "ms_per_step", "steps", "warmup", "dtype", "config", "pct_of_nominal_8TBs", "step_GBps",
+            "bytes_per_step", "stage_ms", "aggregate_path", "roofline", "clocks", "gpu_launches", "verified")
+    for name in reversed(names):
         steps = args.steps if args.steps is not None else DEFAULT_STEPS.get(name, 50)
         warmup = max(3, 5 if args.warmup is None else args.warmup)
-        rec, work, bytes_all = measure(job, name, steps, warmup, full=(i == 0))
-        if i == 0:
+        rec, work, bytes_all = measure(job, name, steps, warmup, full=(name == names[0]))
+        if name == names[0]:
             out = rec
             if job.rank == 0 and job.world == 1 and not args.no_cpu_baseline:
                 out["cpu_baseline"] = cpu_baseline(work)
-            if len(names) > 1:
-                out["per_config"] = []
         else:
-            keep = ("value", "unit", "ms_per_step", "steps", "warmup", "dtype", "config", "pct_of_nominal_8TBs", "step_GBps",
-                    "bytes_per_step", "stage_ms", "aggregate_path", "roofline", "clocks", "gpu_launches", "verified")
-            out["per_config"].append({k: rec[k] for k in keep} | {k: v for k, v in rec.items() if k.startswith("pct_of_")})
+            others.append({k: rec[k] for k in keep} | {k: v for k, v in rec.items() if k.startswith("pct_of_")})
+    if len(names) > 1:
+        out["per_config"] = others
     if left_out:
         out["config"]["left_out"] = "%s: not enough free device memory" % ", ".join(left_out)
     if job.dist is not None:
