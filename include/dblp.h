@@ -358,9 +358,13 @@ int dblp_round_device(const dblp_plan_t* plan, const void* const* grads, const d
                       const dblp_round_marks_t* marks, void* stream);
 
 /* dblp_round_host = the same round from HOST gradients (grads_host: HOST array of W host pointers, pinned memory
- * recommended): worker w's gradient is copied into dev->grads on the plan's copy stream while worker w - 1 is being
- * packetized, the loss process runs beside both, then dblp_round_receive; the aggregate, the counters and the bound
- * outputs are copied back to the host pointers (NULL to skip) and the call waits for the stream.  Nothing is
+ * recommended).  Gradients of 32 MiB per worker and more are taken in up to 16 parts, contiguous ranges of chunks: the
+ * host-to-device copies into dev->grads run back to back on a copy stream of the plan, part by part and worker by
+ * worker; each slice is packetized as soon as it has landed; once a part is there for all workers its packets are
+ * claimed, its chunks reduced, and its range of the aggregate starts back to agg_host on another stream of the plan,
+ * so the copy back overlaps the copies in of the later parts.  The loss process runs beside all of it, the bitmap and
+ * the tolerance test after the last claims.  Results are those of dblp_round_device.  The aggregate, the counters and
+ * the bound outputs are copied back to the host pointers (NULL to skip) and the call waits for all of it.  Nothing is
  * allocated. */
 int dblp_round_host(const dblp_plan_t* plan, const void* const* grads_host, const dblp_loss_model_t* model,
                     uint64_t seed, uint32_t round, uint32_t bound_ppm, uint32_t flags,

@@ -143,8 +143,10 @@ k_book(const dblp_hdr_t* __restrict__ hdr_ring, uint64_t n_slots, const uint32_t
        const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap, uint32_t round,
        unsigned long long* __restrict__ slot_key, dblp_counters_t* counters,
        const uint4* __restrict__ tensor_tab, uint32_t T, uint32_t W, uint64_t C, uint32_t E, uint32_t es,
-       uint32_t hdr_stride)
+       uint32_t hdr_stride, uint32_t part_lo, uint32_t part_hi)
 {
+    // part_hi != 0: this launch is one of several passes over the same arrival list and takes only the entries whose
+    // slot number modulo C lies in [part_lo, part_hi); every entry belongs to exactly one pass, whatever its slot.
     __shared__ uint32_t s_cnt[3];
     const bool wide = ((reinterpret_cast<uintptr_t>(hdr_ring) | hdr_stride) & 31u) == 0;
     const uint64_t n = min(*n_arrived_dev, arrival_cap);
@@ -157,7 +159,11 @@ k_book(const dblp_hdr_t* __restrict__ hdr_ring, uint64_t n_slots, const uint32_t
 #pragma unroll
     for (int k = 0; k < kBookItems; ++k) {
         const uint64_t a = a0 + (uint64_t)k * kBookThreads;
-        if (a < n) { slot[k] = __ldg(&arrival[a]); live |= 1u << k; }
+        if (a < n) {
+            slot[k] = __ldg(&arrival[a]);
+            const uint32_t part = part_hi ? slot[k] % (uint32_t)C : 0u;
+            if (!part_hi || (part >= part_lo && part < part_hi)) live |= 1u << k;
+        }
     }
 #pragma unroll
     for (int k = 0; k < kBookItems; ++k) {
@@ -491,7 +497,8 @@ __device__ __forceinline__ void st_agg32(float* p, const float (&a)[8])
 #endif
 constexpr int kTileThreads = DBLP_REDUCE_THREADS;
 
-// The tile a block sums in its turn-th step (turn = blockIdx.x, blockIdx.x + gridDim.x, ...): the last tile first.
+// The tile (of the n_tiles a launch covers, counted from the launch's first) that a block sums in its turn-th step
+// (turn = blockIdx.x, blockIdx.x + gridDim.x, ...): the last tile first.
 // Right after packetize the most recently written ring slots are the ones still in L2, and those are the last tiles';
 // on a ring a few times the L2 this order was worth 2 % of the reduce's time, on large rings it makes no difference.
 __device__ __forceinline__ uint32_t tile_of_turn(uint32_t turn, uint32_t n_tiles) { return n_tiles - 1 - turn; }
@@ -689,7 +696,7 @@ template <int ES, int WB, int J, bool EXTRA>
 __global__ void __launch_bounds__(kTileThreads, DBLP_REDUCE_MIN_BLOCKS)
 k_reduce_tiled(const uint8_t* __restrict__ ring, const unsigned long long* __restrict__ slot_key,
                const uint64_t* __restrict__ chunk_desc, float* __restrict__ agg, uint32_t W, uint32_t C, uint32_t P,
-               uint32_t VPC, uint32_t CH, uint32_t n_tiles, int mean, float Wf, ReduceExtras ex)
+               uint32_t VPC, uint32_t CH, uint32_t tile_lo, uint32_t n_tiles, int mean, float Wf, ReduceExtras ex)
 {
     constexpr int VE = 16 / ES;
     __shared__ double s_norm[kTileThreads / 32];
@@ -703,11 +710,11 @@ k_reduce_tiled(const uint8_t* __restrict__ ring, const unsigned long long* __res
     auto chunk_of = [&](uint32_t i) { return VPC == 1 ? i : __umulhi(i, vpc_magic); };
 
     uint32_t turn = blockIdx.x, buf = 0;
-    if (turn < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, tile_of_turn(turn, n_tiles), 0, CH, C, W);
+    if (turn < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, tile_lo + tile_of_turn(turn, n_tiles), 0, CH, C, W);
     cp_async_commit();
     for (; turn < n_tiles; turn += gridDim.x, buf ^= 1) {
-        const uint32_t tile = tile_of_turn(turn, n_tiles), next = turn + gridDim.x;
-        if (next < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, tile_of_turn(next, n_tiles), buf ^ 1, CH, C, W);
+        const uint32_t tile = tile_lo + tile_of_turn(turn, n_tiles), next = turn + gridDim.x;
+        if (next < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, tile_lo + tile_of_turn(next, n_tiles), buf ^ 1, CH, C, W);
         cp_async_commit();
         cp_async_wait<1>();                   // everything but the group just committed has landed
         __syncthreads();
@@ -794,7 +801,7 @@ template <int ES, int WB, int S, bool EXTRA>
 __global__ void __launch_bounds__(kTileThreads, (EXTRA && ES == 2 && S == 8) ? 3 : DBLP_REDUCE_MIN_BLOCKS)   // the one shape that needs more than 64 registers
 k_reduce_rows(const uint8_t* __restrict__ ring, const unsigned long long* __restrict__ slot_key,
               const uint64_t* __restrict__ chunk_desc, float* __restrict__ agg, uint32_t W, uint32_t C, uint32_t P,
-              uint32_t CH, uint32_t n_tiles, int mean, float Wf, ReduceExtras ex)
+              uint32_t CH, uint32_t tile_lo, uint32_t n_tiles, int mean, float Wf, ReduceExtras ex)
 {
     constexpr int VE = 16 / ES;
     constexpr uint32_t kWarps = kTileThreads / 32;
@@ -806,11 +813,11 @@ k_reduce_rows(const uint8_t* __restrict__ ring, const unsigned long long* __rest
     const uint2* cells = reinterpret_cast<const uint2*>(slot_key);
 
     uint32_t turn = blockIdx.x, buf = 0;
-    if (turn < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, tile_of_turn(turn, n_tiles), 0, CH, C, W);
+    if (turn < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, tile_lo + tile_of_turn(turn, n_tiles), 0, CH, C, W);
     cp_async_commit();
     for (; turn < n_tiles; turn += gridDim.x, buf ^= 1) {
-        const uint32_t tile = tile_of_turn(turn, n_tiles), next = turn + gridDim.x;
-        if (next < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, tile_of_turn(next, n_tiles), buf ^ 1, CH, C, W);
+        const uint32_t tile = tile_lo + tile_of_turn(turn, n_tiles), next = turn + gridDim.x;
+        if (next < n_tiles) prefetch_tile(sdesc, sslot, cells, chunk_desc, tile_lo + tile_of_turn(next, n_tiles), buf ^ 1, CH, C, W);
         cp_async_commit();
         cp_async_wait<1>();
         __syncthreads();
@@ -901,8 +908,9 @@ k_norm_finish(const double* __restrict__ partials, uint32_t n, double* __restric
 
 template <int ES, int WB, int J>
 static cudaError_t launch_tiled(const dblp_plan* p, const uint8_t* ring, const unsigned long long* slot_key, float* agg,
-                                int mean, const ReduceExtras* ex, cudaStream_t s)
+                                int mean, const ReduceExtras* ex, cudaStream_t s, uint32_t tile_lo, uint32_t n_tiles)
 {
+    const uint32_t grid = p->red_grid < n_tiles ? p->red_grid : n_tiles;
     // sum / (float)W: for W = 1 nothing to do, for a power of two a multiplication by the exact reciprocal gives the
     // identical correctly rounded result, otherwise an IEEE division
     float Wf = (float)p->W;
@@ -912,22 +920,22 @@ static cudaError_t launch_tiled(const dblp_plan* p, const uint8_t* ring, const u
     }
     if (p->red_rows) {
         if (ex)
-            k_reduce_rows<ES, WB, J, true><<<p->red_grid, kTileThreads, p->red_smem, s>>>(
-                ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->pay_stride, p->red_CH, p->red_tiles, mean, Wf,
+            k_reduce_rows<ES, WB, J, true><<<grid, kTileThreads, p->red_smem, s>>>(
+                ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->pay_stride, p->red_CH, tile_lo, n_tiles, mean, Wf,
                 *ex);
         else
-            k_reduce_rows<ES, WB, J, false><<<p->red_grid, kTileThreads, p->red_smem, s>>>(
-                ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->pay_stride, p->red_CH, p->red_tiles, mean, Wf,
+            k_reduce_rows<ES, WB, J, false><<<grid, kTileThreads, p->red_smem, s>>>(
+                ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->pay_stride, p->red_CH, tile_lo, n_tiles, mean, Wf,
                 ReduceExtras{nullptr, nullptr, 0.0f, 0});
         return cudaGetLastError();
     }
     if (ex)
-        k_reduce_tiled<ES, WB, J, true><<<p->red_grid, kTileThreads, p->red_smem, s>>>(
-            ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->pay_stride, p->VPC, p->red_CH, p->red_tiles, mean,
+        k_reduce_tiled<ES, WB, J, true><<<grid, kTileThreads, p->red_smem, s>>>(
+            ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->pay_stride, p->VPC, p->red_CH, tile_lo, n_tiles, mean,
             Wf, *ex);
     else
-        k_reduce_tiled<ES, WB, J, false><<<p->red_grid, kTileThreads, p->red_smem, s>>>(
-            ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->pay_stride, p->VPC, p->red_CH, p->red_tiles, mean,
+        k_reduce_tiled<ES, WB, J, false><<<grid, kTileThreads, p->red_smem, s>>>(
+            ring, slot_key, p->d_chunk_desc, agg, p->W, (uint32_t)p->C, p->pay_stride, p->VPC, p->red_CH, tile_lo, n_tiles, mean,
             Wf, ReduceExtras{nullptr, nullptr, 0.0f, 0});
     return cudaGetLastError();
 }
@@ -939,22 +947,22 @@ static cudaError_t occupancy_tiled(int* blocks, size_t smem)
 }
 
 static void launch_tiled_for(const dblp_plan* plan, const uint8_t* ring, const unsigned long long* keys, float* agg_out,
-                             int mean, const ReduceExtras* ex, cudaStream_t s)
+                             int mean, const ReduceExtras* ex, cudaStream_t s, uint32_t tile_lo, uint32_t n_tiles)
 {
     const int J = plan->red_variant;
     if (J == 8) {
-        if (plan->es == 4) launch_tiled<4, 1, 8>(plan, ring, keys, agg_out, mean, ex, s);
-        else launch_tiled<2, 1, 8>(plan, ring, keys, agg_out, mean, ex, s);
+        if (plan->es == 4) launch_tiled<4, 1, 8>(plan, ring, keys, agg_out, mean, ex, s, tile_lo, n_tiles);
+        else launch_tiled<2, 1, 8>(plan, ring, keys, agg_out, mean, ex, s, tile_lo, n_tiles);
         return;
     }
     if (plan->es == 4) {
-        if (J == 4) launch_tiled<4, 2, 4>(plan, ring, keys, agg_out, mean, ex, s);
-        else if (J == 2 && plan->W <= 4) launch_tiled<4, 4, 2>(plan, ring, keys, agg_out, mean, ex, s);
-        else launch_tiled<4, 8, kJWide>(plan, ring, keys, agg_out, mean, ex, s);
+        if (J == 4) launch_tiled<4, 2, 4>(plan, ring, keys, agg_out, mean, ex, s, tile_lo, n_tiles);
+        else if (J == 2 && plan->W <= 4) launch_tiled<4, 4, 2>(plan, ring, keys, agg_out, mean, ex, s, tile_lo, n_tiles);
+        else launch_tiled<4, 8, kJWide>(plan, ring, keys, agg_out, mean, ex, s, tile_lo, n_tiles);
     } else {
-        if (J == 4) launch_tiled<2, 2, 4>(plan, ring, keys, agg_out, mean, ex, s);
-        else if (J == 2 && plan->W <= 4) launch_tiled<2, 4, 2>(plan, ring, keys, agg_out, mean, ex, s);
-        else launch_tiled<2, 8, kJWide>(plan, ring, keys, agg_out, mean, ex, s);
+        if (J == 4) launch_tiled<2, 2, 4>(plan, ring, keys, agg_out, mean, ex, s, tile_lo, n_tiles);
+        else if (J == 2 && plan->W <= 4) launch_tiled<2, 4, 2>(plan, ring, keys, agg_out, mean, ex, s, tile_lo, n_tiles);
+        else launch_tiled<2, 8, kJWide>(plan, ring, keys, agg_out, mean, ex, s, tile_lo, n_tiles);
     }
 }
 
@@ -1011,9 +1019,11 @@ int configure_reduce(dblp_plan* p, uint32_t ch_override, uint32_t grid_override)
 
 using namespace dblp;
 
-extern "C" int dblp_aggregate_claim(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, uint64_t n_slots,
-                                    const uint32_t* arrival, const uint64_t* n_arrived_dev, uint64_t arrival_cap,
-                                    uint32_t round, uint64_t* slot_key, dblp_counters_t* counters, void* stream)
+namespace dblp {
+
+int claim_arrivals(const dblp_plan* plan, const dblp_hdr_t* hdr_ring, uint64_t n_slots, const uint32_t* arrival,
+                   const uint64_t* n_arrived_dev, uint64_t arrival_cap, uint32_t round, uint64_t* slot_key,
+                   dblp_counters_t* counters, uint32_t part_lo, uint32_t part_hi, cudaStream_t s)
 {
     DBLP_REQUIRE(plan && hdr_ring && arrival && n_arrived_dev && slot_key && counters, DBLP_EINVAL,
                  "aggregate_claim: null argument");
@@ -1022,11 +1032,35 @@ extern "C" int dblp_aggregate_claim(const dblp_plan_t* plan, const dblp_hdr_t* h
     DBLP_REQUIRE(arrival_cap < (1ull << 32), DBLP_ECAPACITY, "aggregate_claim: arrival list too long");
     if (arrival_cap == 0) return DBLP_OK;
     const unsigned grid = (unsigned)((arrival_cap + kBookThreads * kBookItems - 1) / (kBookThreads * kBookItems));
-    k_book<<<grid, kBookThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+    k_book<<<grid, kBookThreads, 0, s>>>(
         hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, reinterpret_cast<unsigned long long*>(slot_key), counters,
-        plan->d_tensor_tab, plan->T, plan->W, plan->C, plan->E, plan->es, plan->hdr_stride);
+        plan->d_tensor_tab, plan->T, plan->W, plan->C, plan->E, plan->es, plan->hdr_stride, part_lo, part_hi);
     DBLP_LAUNCHED();
     return DBLP_OK;
+}
+
+int reduce_chunks(const dblp_plan* plan, const void* payload_ring, const uint64_t* slot_key, float* agg_out, uint32_t flags,
+                  uint64_t chunk_lo, uint64_t chunk_hi, cudaStream_t s)
+{
+    DBLP_REQUIRE(plan->red_variant && chunk_lo % plan->red_CH == 0 && chunk_lo < chunk_hi && chunk_hi <= plan->C &&
+                 (chunk_hi % plan->red_CH == 0 || chunk_hi == plan->C), DBLP_EINVAL,
+                 "reduce_chunks: the range must consist of whole tiles of the tiled reduce");
+    const uint32_t tile_lo = (uint32_t)(chunk_lo / plan->red_CH);
+    const uint32_t n_tiles = (uint32_t)((chunk_hi + plan->red_CH - 1) / plan->red_CH) - tile_lo;
+    launch_tiled_for(plan, static_cast<const uint8_t*>(payload_ring) + plan->pay_off,
+                     reinterpret_cast<const unsigned long long*>(slot_key), agg_out, flags == DBLP_MEAN, nullptr, s, tile_lo, n_tiles);
+    DBLP_LAUNCHED();
+    return DBLP_OK;
+}
+
+}  // namespace dblp
+
+extern "C" int dblp_aggregate_claim(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, uint64_t n_slots,
+                                    const uint32_t* arrival, const uint64_t* n_arrived_dev, uint64_t arrival_cap,
+                                    uint32_t round, uint64_t* slot_key, dblp_counters_t* counters, void* stream)
+{
+    return claim_arrivals(plan, hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, slot_key, counters, 0, 0,
+                          static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int dblp_aggregate_bitmap(const dblp_plan_t* plan, const uint64_t* slot_key, const uint64_t* n_arrived_dev,
@@ -1118,7 +1152,7 @@ extern "C" int dblp_aggregate_reduce(const dblp_plan_t* plan, const void* payloa
     const uint8_t* ring = static_cast<const uint8_t*>(payload_ring) + plan->pay_off;
     const unsigned long long* keys = reinterpret_cast<const unsigned long long*>(slot_key);
     if (plan->red_variant) {
-        launch_tiled_for(plan, ring, keys, agg_out, mean, nullptr, s);
+        launch_tiled_for(plan, ring, keys, agg_out, mean, nullptr, s, 0, plan->red_tiles);
         DBLP_LAUNCHED();
         return DBLP_OK;
     }
@@ -1160,7 +1194,7 @@ extern "C" int dblp_aggregate_reduce_ex(const dblp_plan_t* plan, const void* pay
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const ReduceExtras ex{norm_scratch, params, lr, (flags & DBLP_OUT_BF16) ? 1 : 0};
     launch_tiled_for(plan, static_cast<const uint8_t*>(payload_ring) + plan->pay_off, reinterpret_cast<const unsigned long long*>(slot_key),
-                     agg_out, (flags & DBLP_MEAN) ? 1 : 0, &ex, s);
+                     agg_out, (flags & DBLP_MEAN) ? 1 : 0, &ex, s, 0, plan->red_tiles);
     DBLP_LAUNCHED();
     if (norm_scratch) {
         k_norm_finish<<<1, 1024, 0, s>>>(norm_scratch, plan->red_tiles, norm_out);

@@ -108,8 +108,8 @@ struct dblp_plan {
     // Host-side resources of the whole-round calls (round.cu): a high-priority stream for the work that runs beside
     // the two bandwidth-bound kernels, a stream for host-to-device copies, and the events that order them.  They make
     // a plan serve one whole-round call at a time.
-    cudaStream_t side, copy;
-    cudaEvent_t ev_fork, ev_join, ev_claimed, ev_done, ev_copy[2];
+    cudaStream_t side, copy, back;
+    cudaEvent_t ev_fork, ev_join, ev_claimed, ev_done, ev_copy[2], ev_part[2], ev_back;
     // launch shape of the masked reduce (configure_reduce): red_variant = items per thread of the tiled kernel,
     // 0 = the simple one-vector-per-thread kernel
     uint32_t red_variant, red_CH, red_tiles, red_grid, red_rows;
@@ -126,7 +126,17 @@ struct dblp_plan {
 
 namespace dblp {
 int configure_reduce(dblp_plan* p, uint32_t ch_override, uint32_t grid_override);
-// dblp_packetize for workers w0 .. w0 + nw - 1 only; grads[k] is worker (w0 + k)'s gradient.
+// dblp_packetize for workers w0 .. w0 + nw - 1 and chunks chunk_lo .. chunk_hi - 1 only; grads[k] is worker (w0 + k)'s
+// whole gradient.
 int packetize_workers(const dblp_plan* plan, const void* const* grads, uint32_t w0, uint32_t nw, uint32_t round,
-                      dblp_hdr_t* hdr_ring, void* payload_ring, cudaStream_t s);
+                      dblp_hdr_t* hdr_ring, void* payload_ring, uint64_t chunk_lo, uint64_t chunk_hi, cudaStream_t s);
+// dblp_aggregate_claim, optionally as one of several passes over the arrival list: with part_hi != 0 only the entries
+// whose slot number modulo C lies in [part_lo, part_hi) are examined (and counted); part_hi = 0 takes all.
+int claim_arrivals(const dblp_plan* plan, const dblp_hdr_t* hdr_ring, uint64_t n_slots, const uint32_t* arrival,
+                   const uint64_t* n_arrived_dev, uint64_t arrival_cap, uint32_t round, uint64_t* slot_key,
+                   dblp_counters_t* counters, uint32_t part_lo, uint32_t part_hi, cudaStream_t s);
+// dblp_aggregate_reduce for chunks chunk_lo .. chunk_hi - 1 (whole tiles of the tiled reduce: chunk_lo a multiple of
+// red_CH, chunk_hi a multiple of it or C); needs red_variant != 0.
+int reduce_chunks(const dblp_plan* plan, const void* payload_ring, const uint64_t* slot_key, float* agg_out, uint32_t flags,
+                  uint64_t chunk_lo, uint64_t chunk_hi, cudaStream_t s);
 }

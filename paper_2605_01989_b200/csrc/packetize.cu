@@ -47,8 +47,8 @@ __device__ __forceinline__ void st_keep16(void* p, uint4 v)
 
 template <int ES>
 __global__ void __launch_bounds__(kPackThreads)
-k_packetize(GradPtrs grads, uint32_t w0, uint32_t nw_fast, uint32_t C, uint32_t VPC, uint32_t pay_stride, uint32_t hdr_stride, uint32_t CH,
-            uint32_t round,
+k_packetize(GradPtrs grads, uint32_t w0, uint32_t nw_fast, uint32_t c_lo, uint32_t c_hi, uint32_t C, uint32_t VPC,
+            uint32_t pay_stride, uint32_t hdr_stride, uint32_t CH, uint32_t round,
             const uint64_t* __restrict__ chunk_desc, const uint32_t* __restrict__ chunk_tensor,
             const uint64_t* __restrict__ tensor_base, dblp_hdr_t* __restrict__ hdr_ring, uint8_t* __restrict__ ring)
 {
@@ -61,7 +61,7 @@ k_packetize(GradPtrs grads, uint32_t w0, uint32_t nw_fast, uint32_t C, uint32_t 
     }
     const uint32_t w = w0 + wl, tid = threadIdx.x;
     const uint8_t* __restrict__ g = static_cast<const uint8_t*>(grads.p[wl]);
-    const uint32_t c0 = tile * CH, nch = min(CH, C - c0);
+    const uint32_t c0 = c_lo + tile * CH, nch = min(CH, c_hi - c0);     // the launch covers chunks c_lo .. c_hi - 1
     const uint64_t slot0 = (uint64_t)w * C + c0;
 
     for (uint32_t k = tid; k < nch; k += kPackThreads) {
@@ -115,11 +115,12 @@ k_packetize(GradPtrs grads, uint32_t w0, uint32_t nw_fast, uint32_t C, uint32_t 
 }
 
 int packetize_workers(const dblp_plan* plan, const void* const* grads, uint32_t w_first, uint32_t n_workers, uint32_t round,
-                      dblp_hdr_t* hdr_ring, void* payload_ring, cudaStream_t s)
+                      dblp_hdr_t* hdr_ring, void* payload_ring, uint64_t chunk_lo, uint64_t chunk_hi, cudaStream_t s)
 {
+    DBLP_REQUIRE(chunk_lo < chunk_hi && chunk_hi <= plan->C, DBLP_EINVAL, "packetize: empty or out-of-range chunk range");
     uint32_t CH = (4096u + plan->VPC - 1) / plan->VPC;          // about 64 KB of payload per block
     if (CH > kPackMaxTile) CH = kPackMaxTile;
-    const uint64_t gx = (plan->C + CH - 1) / CH;
+    const uint64_t gx = (chunk_hi - chunk_lo + CH - 1) / CH;
     DBLP_REQUIRE(gx * kMaxWorkersPerLaunch < (1ull << 31), DBLP_ECAPACITY, "packetize: grid too large");
     for (uint32_t w0 = w_first; w0 < w_first + n_workers; w0 += kMaxWorkersPerLaunch) {
         const uint32_t nw = min(kMaxWorkersPerLaunch, w_first + n_workers - w0);
@@ -128,10 +129,10 @@ int packetize_workers(const dblp_plan* plan, const void* const* grads, uint32_t 
         const uint32_t nw_fast = plan->pack_tile_major ? nw : 0u;
         const dim3 grid = nw_fast ? dim3((unsigned)(gx * nw), 1) : dim3((unsigned)gx, nw);
         if (plan->es == 4)
-            k_packetize<4><<<grid, kPackThreads, 0, s>>>(gp, w0, nw_fast, (uint32_t)plan->C, plan->VPC, plan->pay_stride, plan->hdr_stride, CH, round,
+            k_packetize<4><<<grid, kPackThreads, 0, s>>>(gp, w0, nw_fast, (uint32_t)chunk_lo, (uint32_t)chunk_hi, (uint32_t)plan->C, plan->VPC, plan->pay_stride, plan->hdr_stride, CH, round,
                 plan->d_chunk_desc, plan->d_chunk_tensor, plan->d_base, hdr_ring, static_cast<uint8_t*>(payload_ring) + plan->pay_off);
         else
-            k_packetize<2><<<grid, kPackThreads, 0, s>>>(gp, w0, nw_fast, (uint32_t)plan->C, plan->VPC, plan->pay_stride, plan->hdr_stride, CH, round,
+            k_packetize<2><<<grid, kPackThreads, 0, s>>>(gp, w0, nw_fast, (uint32_t)chunk_lo, (uint32_t)chunk_hi, (uint32_t)plan->C, plan->VPC, plan->pay_stride, plan->hdr_stride, CH, round,
                 plan->d_chunk_desc, plan->d_chunk_tensor, plan->d_base, hdr_ring, static_cast<uint8_t*>(payload_ring) + plan->pay_off);
         DBLP_LAUNCHED();
     }
@@ -152,5 +153,5 @@ extern "C" int dblp_packetize(const dblp_plan_t* plan, const void* const* grads,
         DBLP_REQUIRE((reinterpret_cast<uintptr_t>(grads[w]) % plan->es) == 0, DBLP_EALIGN,
                      "packetize: gradient of worker %u is not element-aligned", w);
     }
-    return packetize_workers(plan, grads, 0, plan->W, round, hdr_ring, payload_ring, static_cast<cudaStream_t>(stream));
+    return packetize_workers(plan, grads, 0, plan->W, round, hdr_ring, payload_ring, 0, plan->C, static_cast<cudaStream_t>(stream));
 }

@@ -32,7 +32,9 @@ static void free_tables(dblp_plan* p)
     cudaFree(p->d_ticket);
     if (p->side) cudaStreamDestroy(p->side);
     if (p->copy) cudaStreamDestroy(p->copy);
-    cudaEvent_t* evs[] = {&p->ev_fork, &p->ev_join, &p->ev_claimed, &p->ev_done, &p->ev_copy[0], &p->ev_copy[1]};
+    if (p->back) cudaStreamDestroy(p->back);
+    cudaEvent_t* evs[] = {&p->ev_fork, &p->ev_join,    &p->ev_claimed, &p->ev_done, &p->ev_copy[0],
+                          &p->ev_copy[1], &p->ev_part[0], &p->ev_part[1], &p->ev_back};
     for (cudaEvent_t* e : evs)
         if (*e) cudaEventDestroy(*e);
 }
@@ -45,7 +47,9 @@ static cudaError_t create_round_resources(dblp_plan* p)
     cudaError_t e = cudaDeviceGetStreamPriorityRange(&least, &greatest);
     if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&p->side, cudaStreamNonBlocking, greatest);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->copy, cudaStreamNonBlocking);
-    cudaEvent_t* evs[] = {&p->ev_fork, &p->ev_join, &p->ev_claimed, &p->ev_done, &p->ev_copy[0], &p->ev_copy[1]};
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->back, cudaStreamNonBlocking);
+    cudaEvent_t* evs[] = {&p->ev_fork, &p->ev_join,    &p->ev_claimed, &p->ev_done, &p->ev_copy[0],
+                          &p->ev_copy[1], &p->ev_part[0], &p->ev_part[1], &p->ev_back};
     for (cudaEvent_t* ev : evs)
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
     return e;
@@ -87,8 +91,9 @@ static int plan_create(const uint64_t* tensor_numel, uint32_t T, int dtype, uint
     p->hdr_stride = 32; p->pay_stride = payload_bytes; p->pay_off = 0;
     p->d_tensor_tab = nullptr; p->d_base = nullptr; p->d_chunk_desc = nullptr;
     p->d_chunk_tensor = p->d_bucket_bounds = p->d_bound_ppm = p->d_ticket = nullptr;
-    p->side = p->copy = nullptr;
+    p->side = p->copy = p->back = nullptr;
     p->ev_fork = p->ev_join = p->ev_claimed = p->ev_done = p->ev_copy[0] = p->ev_copy[1] = nullptr;
+    p->ev_part[0] = p->ev_part[1] = p->ev_back = nullptr;
 
     uint64_t base = 0, c = 0;
     p->h_numel.assign(tensor_numel, tensor_numel + T);

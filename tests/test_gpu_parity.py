@@ -276,34 +276,60 @@ def test_datagram_wire_format(dtype, P):
     g.close()
 
 
-def test_round_host_entry_point_matches_the_oracle():
-    w = work(RAGGED, "f32", 1408, 3, wl.LossSpec("ge", 0.05, 6.0), 41)
-    op = orc.Plan(w.numel, 4, 1408, 3)
+def _round_host_parity(w, bound_ppm=60000, reps=2):
+    """dblp_round_host on workload w, `reps` calls in a row on the same buffers: everything it hands back to the host
+    and the state it leaves on the device, against the oracle."""
+    op = orc.Plan(w.numel, w.elem_size, w.payload_bytes, w.W)
     gm, om = H.models_for(w, op.C)
     grads_host = [x.pin_memory() for x in wl.make_grads(w, "cpu")]
     g = H.GpuRound(w)
-    grads_dev = torch.empty(w.W * w.N, dtype=torch.float32, device=H.DEV)
+    grads_dev = torch.empty(w.W * w.N, dtype=grads_host[0].dtype, device=H.DEV)
     agg_host = torch.empty(w.N, dtype=torch.float32).pin_memory()
     cnt_host = torch.zeros(7, dtype=torch.int64).pin_memory()
-    recv_host = torch.zeros(3, dtype=torch.int32).pin_memory()
-    miss_host = torch.zeros(3, dtype=torch.int32).pin_memory()
-    ok_host = torch.zeros(3, dtype=torch.uint8).pin_memory()
+    recv_host = torch.zeros(w.W, dtype=torch.int32).pin_memory()
+    miss_host = torch.zeros(w.W, dtype=torch.int32).pin_memory()
+    ok_host = torch.zeros(w.W, dtype=torch.uint8).pin_memory()
     all_host = torch.zeros(1, dtype=torch.int32).pin_memory()
-    for rep in range(2):                       # second call reuses every buffer
-        dblp.dblp_round_host(g.plan, grads_host, gm, w.seed, w.round + rep, 60000, dblp.DBLP_MEAN, g.buf, grads_dev,
+    host = H.to_host(grads_host, w.dtype)
+    for rep in range(reps):                    # later calls reuse every buffer
+        rnd = w.round + rep
+        agg_host.fill_(float("nan"))
+        dblp.dblp_round_host(g.plan, grads_host, gm, w.seed, rnd, bound_ppm, dblp.DBLP_MEAN, g.buf, grads_dev,
                              agg_host, cnt_host, recv_host, miss_host, ok_host, all_host)
-        host = [x.numpy() for x in grads_host]
-        o_hdr, o_pay = op.packetize(host, w.round + rep)
-        o_del, _ = op.loss_mask(om, w.seed, w.round + rep)
-        o_arr, o_n = op.arrival(o_del, w.seed, w.round + rep)
-        st = op.book(o_hdr, o_arr, o_n, w.round + rep, op.new_state())
-        H.assert_bits_equal(agg_host.numpy(), op.reduce(o_pay, st, mean=True), "aggregate via round_host")
-        o = op.check_bound(st["bitmap"], 60000)
+        o_hdr, o_pay = op.packetize(host, rnd)
+        o_del, _ = op.loss_mask(om, w.seed, rnd)
+        o_arr, o_n = op.arrival(o_del, w.seed, rnd)
+        st = op.book(o_hdr, o_arr, o_n, rnd, op.new_state())
+        want = op.reduce(o_pay, st, mean=True)
+        H.assert_bits_equal(agg_host.numpy(), want, "aggregate via round_host")
+        H.assert_bits_equal(g.buf["agg"].cpu().numpy(), want, "aggregate left on the device")
+        H.assert_bits_equal(H.hdr_np(g.buf["hdr_ring"]), o_hdr, "header ring")
+        assert g.buf["payload_ring"].cpu().numpy().tobytes() == o_pay.tobytes(), "payload ring"
+        H.compare_state(g, st, op)
+        o = op.check_bound(st["bitmap"], bound_ppm)
         assert recv_host.numpy().view(np.uint32).tolist() == o[0][:, 0].tolist()
         assert miss_host.numpy().view(np.uint32).tolist() == o[1][:, 0].tolist()
         assert ok_host.numpy().tolist() == o[2][:, 0].tolist() and int(all_host[0]) == o[3]
         assert dict(zip(dblp.COUNTER_FIELDS, cnt_host.tolist()[:6])) == st["counters"].as_dict()
     g.close()
+
+
+def test_round_host_entry_point_matches_the_oracle():
+    _round_host_parity(work(RAGGED, "f32", 1408, 3, wl.LossSpec("ge", 0.05, 6.0), 41))
+
+
+@pytest.mark.parametrize("name,w", [
+    ("resnet50: six parts", wl.config(1)),
+    ("sixteen parts that cut through tensors, fp32", work([40_000_003, 17, 90_000_001, 4096 * 3 + 5], "f32", 4096, 2,
+                                                        wl.LossSpec("iid", 0.03), 43)),
+    ("sixteen parts, bf16, short payloads", work([100_000_001, 3, 70_000_000], "bf16", 1408, 2,
+                                             wl.LossSpec("ge", 0.05, 6.0), 44)),
+], ids=["resnet50", "f32-many-parts", "bf16-many-parts"])
+def test_round_host_in_several_parts_matches_the_oracle(name, w):
+    """Gradients of 32 MiB and more per worker go through dblp_round_host part by part (copy in, packetize, claim,
+    reduce, copy out, pipelined): the results must be those of the unsplit round."""
+    assert w.N * w.elem_size > (64 << 20)
+    _round_host_parity(w, bound_ppm=w.bounds_ppm[0], reps=2)
 
 
 def test_round_device_schedule_on_the_resnet50_shaped_workload():
