@@ -138,6 +138,7 @@ __device__ __forceinline__ void block_sum3(uint32_t a, uint32_t b, uint32_t c, u
 #endif
 constexpr int kBookItems = DBLP_BOOK_ITEMS;
 
+template <bool PART>
 __global__ void __launch_bounds__(kBookThreads)
 k_book(const dblp_hdr_t* __restrict__ hdr_ring, uint64_t n_slots, const uint32_t* __restrict__ arrival,
        const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap, uint32_t round,
@@ -145,8 +146,8 @@ k_book(const dblp_hdr_t* __restrict__ hdr_ring, uint64_t n_slots, const uint32_t
        const uint4* __restrict__ tensor_tab, uint32_t T, uint32_t W, uint64_t C, uint32_t E, uint32_t es,
        uint32_t hdr_stride, uint32_t part_lo, uint32_t part_hi)
 {
-    // part_hi != 0: this launch is one of several passes over the same arrival list and takes only the entries whose
-    // slot number modulo C lies in [part_lo, part_hi); every entry belongs to exactly one pass, whatever its slot.
+    // PART: this launch is one of several passes over the same arrival list and takes only the entries whose slot
+    // number modulo C lies in [part_lo, part_hi); every entry belongs to exactly one pass, whatever its slot.
     __shared__ uint32_t s_cnt[3];
     const bool wide = ((reinterpret_cast<uintptr_t>(hdr_ring) | hdr_stride) & 31u) == 0;
     const uint64_t n = min(*n_arrived_dev, arrival_cap);
@@ -161,8 +162,12 @@ k_book(const dblp_hdr_t* __restrict__ hdr_ring, uint64_t n_slots, const uint32_t
         const uint64_t a = a0 + (uint64_t)k * kBookThreads;
         if (a < n) {
             slot[k] = __ldg(&arrival[a]);
-            const uint32_t part = part_hi ? slot[k] % (uint32_t)C : 0u;
-            if (!part_hi || (part >= part_lo && part < part_hi)) live |= 1u << k;
+            if (PART) {
+                const uint32_t part = slot[k] % (uint32_t)C;
+                if (part >= part_lo && part < part_hi) live |= 1u << k;
+            } else {
+                live |= 1u << k;
+            }
         }
     }
 #pragma unroll
@@ -1032,9 +1037,15 @@ int claim_arrivals(const dblp_plan* plan, const dblp_hdr_t* hdr_ring, uint64_t n
     DBLP_REQUIRE(arrival_cap < (1ull << 32), DBLP_ECAPACITY, "aggregate_claim: arrival list too long");
     if (arrival_cap == 0) return DBLP_OK;
     const unsigned grid = (unsigned)((arrival_cap + kBookThreads * kBookItems - 1) / (kBookThreads * kBookItems));
-    k_book<<<grid, kBookThreads, 0, s>>>(
-        hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, reinterpret_cast<unsigned long long*>(slot_key), counters,
-        plan->d_tensor_tab, plan->T, plan->W, plan->C, plan->E, plan->es, plan->hdr_stride, part_lo, part_hi);
+    unsigned long long* keys = reinterpret_cast<unsigned long long*>(slot_key);
+    if (part_hi)
+        k_book<true><<<grid, kBookThreads, 0, s>>>(hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, keys, counters,
+                                                   plan->d_tensor_tab, plan->T, plan->W, plan->C, plan->E, plan->es,
+                                                   plan->hdr_stride, part_lo, part_hi);
+    else
+        k_book<false><<<grid, kBookThreads, 0, s>>>(hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, keys, counters,
+                                                    plan->d_tensor_tab, plan->T, plan->W, plan->C, plan->E, plan->es,
+                                                    plan->hdr_stride, 0, 0);
     DBLP_LAUNCHED();
     return DBLP_OK;
 }
