@@ -75,7 +75,7 @@ EXPORTS = ("dblp_plan_create", "dblp_plan_destroy", "dblp_plan_query", "dblp_pla
            "dblp_apply_loss_resend", "dblp_missing_bits", "dblp_stop_workspace_bytes", "dblp_aggregate_book_stop",
            "dblp_round_until_stop",
            "dblp_aggregate_book",
-           "dblp_aggregate_claim", "dblp_aggregate_bitmap", "dblp_aggregate_reduce", "dblp_aggregate_reduce_ex", "dblp_aggregate_reduce_atomic", "dblp_norm_scratch_count", "dblp_aggregate", "dblp_round_reset", "dblp_check_bound", "dblp_bound_ok", "dblp_clr",
+           "dblp_aggregate_claim", "dblp_aggregate_claim_grouped", "dblp_claim_workspace_bytes", "dblp_aggregate_bitmap", "dblp_aggregate_reduce", "dblp_aggregate_reduce_ex", "dblp_aggregate_reduce_atomic", "dblp_norm_scratch_count", "dblp_aggregate", "dblp_round_reset", "dblp_check_bound", "dblp_bound_ok", "dblp_clr",
            "dblp_select_bound", "dblp_round_send", "dblp_round_receive", "dblp_round_device", "dblp_round_host",
            "dblp_strerror", "dblp_last_error", "dblp_launch_count")
 
@@ -192,7 +192,10 @@ class Plan:
         cap = self.M if arrival_cap is None else arrival_cap
         stop_ws = C.c_size_t()
         _check(lib().dblp_stop_workspace_bytes(self.handle, C.c_uint64(cap), C.byref(stop_ws)), "dblp_stop_workspace_bytes")
-        ws_bytes = max(self.workspace_bytes, int(stop_ws.value))
+        claim_ws = C.c_size_t()
+        _check(lib().dblp_claim_workspace_bytes(self.handle, C.c_uint64(n_slots), C.c_uint64(cap), C.byref(claim_ws)),
+               "dblp_claim_workspace_bytes")
+        ws_bytes = max(self.workspace_bytes, int(stop_ws.value), int(claim_ws.value))
         u8, u32, i64 = torch.uint8, torch.int32, torch.int64
         z = lambda n, dt: torch.zeros(n, dtype=dt, device=device)
         return {
@@ -285,6 +288,14 @@ def dblp_aggregate_claim(plan, hdr_ring, n_slots, arrival, n_arrived_dev, arriva
     _check(lib().dblp_aggregate_claim(plan.handle, _ptr(hdr_ring), C.c_uint64(n_slots), _ptr(arrival), _ptr(n_arrived_dev),
                                       C.c_uint64(arrival_cap), C.c_uint32(round), _ptr(slot_key), _ptr(counters),
                                       _stream(stream)), "dblp_aggregate_claim")
+
+
+def dblp_aggregate_claim_grouped(plan, hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, slot_key, counters,
+                                 ws, stream=None):
+    _check(lib().dblp_aggregate_claim_grouped(plan.handle, _ptr(hdr_ring), C.c_uint64(n_slots), _ptr(arrival),
+                                              _ptr(n_arrived_dev), C.c_uint64(arrival_cap), C.c_uint32(round), _ptr(slot_key),
+                                              _ptr(counters), _ptr(ws), C.c_size_t(ws.numel() * ws.element_size()),
+                                              _stream(stream)), "dblp_aggregate_claim_grouped")
 
 
 def dblp_aggregate_bitmap(plan, slot_key, n_arrived_dev, arrival_cap, recv_bitmap, counters, stream=None):

@@ -138,7 +138,9 @@ __device__ __forceinline__ void block_sum3(uint32_t a, uint32_t b, uint32_t c, u
 #endif
 constexpr int kBookItems = DBLP_BOOK_ITEMS;
 
-template <bool PART>
+enum : int { kBookPlain = 0, kBookPart = 1, kBookPairs = 2 };
+
+template <int MODE>
 __global__ void __launch_bounds__(kBookThreads)
 k_book(const dblp_hdr_t* __restrict__ hdr_ring, uint64_t n_slots, const uint32_t* __restrict__ arrival,
        const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap, uint32_t round,
@@ -146,27 +148,37 @@ k_book(const dblp_hdr_t* __restrict__ hdr_ring, uint64_t n_slots, const uint32_t
        const uint4* __restrict__ tensor_tab, uint32_t T, uint32_t W, uint64_t C, uint32_t E, uint32_t es,
        uint32_t hdr_stride, uint32_t part_lo, uint32_t part_hi)
 {
-    // PART: this launch is one of several passes over the same arrival list and takes only the entries whose slot
+    // kBookPart: this launch is one of several passes over the same arrival list and takes only the entries whose slot
     // number modulo C lies in [part_lo, part_hi); every entry belongs to exactly one pass, whatever its slot.
+    // kBookPairs: `arrival` holds 64-bit pairs (position in the arrival list << 32 | slot) in any order (the list after
+    // k_part_scatter has grouped it by slot range), so the arrival number comes from the pair, not from the thread.
     __shared__ uint32_t s_cnt[3];
     const bool wide = ((reinterpret_cast<uintptr_t>(hdr_ring) | hdr_stride) & 31u) == 0;
     const uint64_t n = min(*n_arrived_dev, arrival_cap);
     const uint64_t a0 = (uint64_t)blockIdx.x * (kBookThreads * kBookItems) + threadIdx.x;
     if ((uint64_t)blockIdx.x * (kBookThreads * kBookItems) >= n) return;   // whole block past the end
     const uint64_t first_number = counters->n_arrived;             // arrival numbers continue across calls of a round
-    uint32_t slot[kBookItems];
+    uint32_t slot[kBookItems], pos[kBookItems];                    // pos: the entry's position in the arrival list
     uint4 h0[kBookItems], h1[kBookItems], tt[kBookItems];
     uint32_t live = 0, n_current = 0, n_stale = 0, n_invalid = 0;  // live bit k: item k is still a candidate
 #pragma unroll
     for (int k = 0; k < kBookItems; ++k) {
         const uint64_t a = a0 + (uint64_t)k * kBookThreads;
         if (a < n) {
-            slot[k] = __ldg(&arrival[a]);
-            if (PART) {
-                const uint32_t part = slot[k] % (uint32_t)C;
-                if (part >= part_lo && part < part_hi) live |= 1u << k;
-            } else {
+            if (MODE == kBookPairs) {
+                const uint2 pr = __ldg(reinterpret_cast<const uint2*>(arrival) + a);
+                slot[k] = pr.x;
+                pos[k] = pr.y;
                 live |= 1u << k;
+            } else {
+                slot[k] = __ldg(&arrival[a]);
+                pos[k] = (uint32_t)a;
+                if (MODE == kBookPart) {
+                    const uint32_t part = slot[k] % (uint32_t)C;
+                    if (part >= part_lo && part < part_hi) live |= 1u << k;
+                } else {
+                    live |= 1u << k;
+                }
             }
         }
     }
@@ -189,8 +201,7 @@ k_book(const dblp_hdr_t* __restrict__ hdr_ring, uint64_t n_slots, const uint32_t
         else if (h0[k].y != round) ++n_stale;
         else {
             ++n_current;
-            const uint64_t a = a0 + (uint64_t)k * kBookThreads;
-            atomicMin(&slot_key[(uint64_t)h1[k].z * C + h0[k].x], ((first_number + a) << 32) | slot[k]);
+            atomicMin(&slot_key[(uint64_t)h1[k].z * C + h0[k].x], ((first_number + pos[k]) << 32) | slot[k]);
         }
     }
     block_sum3(n_current, n_stale, n_invalid, s_cnt);
@@ -199,6 +210,109 @@ k_book(const dblp_hdr_t* __restrict__ hdr_ring, uint64_t n_slots, const uint32_t
         if (s_cnt[1]) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_stale), (unsigned long long)s_cnt[1]);
         if (s_cnt[2]) atomicAdd(reinterpret_cast<unsigned long long*>(&counters->n_invalid), (unsigned long long)s_cnt[2]);
     }
+}
+
+// ------------------------------------------------------------------------------------------------ grouping the arrivals
+// Once the headers and the claim table no longer fit in L2, a claim in arrival (that is, random) order costs two
+// random DRAM sectors per packet and the stage runs at what DRAM gives random sectors (12 M packets: 0.54 ms).  Grouping
+// the arrival list by slot range first -- kPartBuckets ranges of 2^shift slots, a counting sort in three small passes
+// whose output is (position, slot) pairs -- makes the claim kernel walk one range's headers and cells at a time, which
+// L2 holds: 0.20 ms for the same 12 M packets plus the passes.  The order inside a range is whatever the scatter's
+// shared-memory atomics give; it does not matter, because the claims are atomic minima over arrival numbers that
+// travel with the pairs.
+constexpr int kPartBuckets = 64;
+constexpr int kPartChunk = 4096;     // arrival entries per block of the counting and scatter passes
+constexpr int kPartThreads = 512;
+
+__device__ __forceinline__ uint32_t part_bucket(uint32_t slot, uint32_t shift)
+{
+    return min(slot >> shift, (uint32_t)kPartBuckets - 1u);       // slot numbers outside the ring land in the last range
+}
+
+__global__ void __launch_bounds__(kPartThreads)
+k_part_count(const uint32_t* __restrict__ arrival, const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap,
+             uint32_t shift, uint32_t* __restrict__ block_hist)
+{
+    __shared__ uint32_t s_hist[kPartBuckets];
+    if (threadIdx.x < kPartBuckets) s_hist[threadIdx.x] = 0;
+    __syncthreads();
+    const uint64_t n = min(*n_arrived_dev, arrival_cap), base = (uint64_t)blockIdx.x * kPartChunk;
+    for (uint32_t k = threadIdx.x; k < kPartChunk; k += kPartThreads) {
+        const uint64_t a = base + k;
+        if (a < n) atomicAdd(&s_hist[part_bucket(__ldg(&arrival[a]), shift)], 1u);
+    }
+    __syncthreads();
+    if (threadIdx.x < kPartBuckets) block_hist[(uint64_t)threadIdx.x * gridDim.x + blockIdx.x] = s_hist[threadIdx.x];   // [range][block]
+}
+
+// One block per range: the range's per-block counts (a contiguous row of the table) become exclusive prefix sums, and
+// the row's total goes to range_total.  The scatter adds the totals of the ranges in front.
+__global__ void __launch_bounds__(1024)
+k_part_offsets(uint32_t* __restrict__ block_hist, uint32_t n_blocks, uint32_t* __restrict__ range_total)
+{
+    __shared__ uint32_t s_scan[1024];
+    uint32_t* row = block_hist + (uint64_t)blockIdx.x * n_blocks;
+    const uint32_t per = (n_blocks + 1023) / 1024;
+    const uint32_t lo = min(n_blocks, threadIdx.x * per), hi = min(n_blocks, lo + per);
+    uint32_t sum = 0;
+    for (uint32_t i = lo; i < hi; ++i) sum += row[i];
+    s_scan[threadIdx.x] = sum;
+    __syncthreads();
+    for (int d = 1; d < 1024; d <<= 1) {
+        const uint32_t v = threadIdx.x >= (uint32_t)d ? s_scan[threadIdx.x - d] : 0;
+        __syncthreads();
+        s_scan[threadIdx.x] += v;
+        __syncthreads();
+    }
+    uint32_t run = s_scan[threadIdx.x] - sum;
+    for (uint32_t i = lo; i < hi; ++i) {
+        const uint32_t c = row[i];
+        row[i] = run;
+        run += c;
+    }
+    if (threadIdx.x == 1023) range_total[blockIdx.x] = s_scan[1023];
+}
+
+__global__ void __launch_bounds__(kPartThreads)
+k_part_scatter(const uint32_t* __restrict__ arrival, const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap,
+               uint32_t shift, const uint32_t* __restrict__ block_off, const uint32_t* __restrict__ range_total,
+               uint2* __restrict__ pairs)
+{
+    __shared__ uint32_t s_cursor[kPartBuckets];
+    if (threadIdx.x < kPartBuckets) {
+        uint32_t first = 0;                                          // where this thread's range starts in the pair list
+        for (uint32_t b = 0; b < threadIdx.x; ++b) first += __ldg(&range_total[b]);
+        s_cursor[threadIdx.x] = first + block_off[(uint64_t)threadIdx.x * gridDim.x + blockIdx.x];
+    }
+    __syncthreads();
+    const uint64_t n = min(*n_arrived_dev, arrival_cap), base = (uint64_t)blockIdx.x * kPartChunk;
+    for (uint32_t k = threadIdx.x; k < kPartChunk; k += kPartThreads) {
+        const uint64_t a = base + k;
+        if (a < n) {
+            const uint32_t slot = __ldg(&arrival[a]);
+            const uint32_t at = atomicAdd(&s_cursor[part_bucket(slot, shift)], 1u);
+            pairs[at] = make_uint2(slot, (uint32_t)a);
+        }
+    }
+}
+
+struct PartLayout {
+    size_t pairs, hist, totals, total;
+    uint32_t n_blocks, shift;
+};
+
+static PartLayout part_layout(uint64_t n_slots, uint64_t arrival_cap)
+{
+    PartLayout l{};
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    l.n_blocks = (uint32_t)((arrival_cap + kPartChunk - 1) / kPartChunk);
+    l.shift = 0;
+    while (n_slots > 0 && ((n_slots - 1) >> l.shift) >= (uint64_t)kPartBuckets) ++l.shift;
+    l.pairs = 0;
+    l.hist = up(arrival_cap * sizeof(uint2));
+    l.totals = up(l.hist + (size_t)l.n_blocks * kPartBuckets * sizeof(uint32_t));
+    l.total = up(l.totals + kPartBuckets * sizeof(uint32_t));
+    return l;
 }
 
 // Rewrites the received bitmap from the claim table (warp ballot -> one word per warp) and folds this call's arrival
@@ -1039,13 +1153,13 @@ int claim_arrivals(const dblp_plan* plan, const dblp_hdr_t* hdr_ring, uint64_t n
     const unsigned grid = (unsigned)((arrival_cap + kBookThreads * kBookItems - 1) / (kBookThreads * kBookItems));
     unsigned long long* keys = reinterpret_cast<unsigned long long*>(slot_key);
     if (part_hi)
-        k_book<true><<<grid, kBookThreads, 0, s>>>(hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, keys, counters,
-                                                   plan->d_tensor_tab, plan->T, plan->W, plan->C, plan->E, plan->es,
-                                                   plan->hdr_stride, part_lo, part_hi);
+        k_book<kBookPart><<<grid, kBookThreads, 0, s>>>(hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, keys,
+                                                        counters, plan->d_tensor_tab, plan->T, plan->W, plan->C, plan->E,
+                                                        plan->es, plan->hdr_stride, part_lo, part_hi);
     else
-        k_book<false><<<grid, kBookThreads, 0, s>>>(hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, keys, counters,
-                                                    plan->d_tensor_tab, plan->T, plan->W, plan->C, plan->E, plan->es,
-                                                    plan->hdr_stride, 0, 0);
+        k_book<kBookPlain><<<grid, kBookThreads, 0, s>>>(hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, keys,
+                                                         counters, plan->d_tensor_tab, plan->T, plan->W, plan->C, plan->E,
+                                                         plan->es, plan->hdr_stride, 0, 0);
     DBLP_LAUNCHED();
     return DBLP_OK;
 }
@@ -1065,6 +1179,47 @@ int reduce_chunks(const dblp_plan* plan, const void* payload_ring, const uint64_
 }
 
 }  // namespace dblp
+
+extern "C" int dblp_claim_workspace_bytes(const dblp_plan_t* plan, uint64_t n_slots, uint64_t arrival_cap, size_t* bytes)
+{
+    DBLP_REQUIRE(plan && bytes, DBLP_EINVAL, "claim_workspace_bytes: null argument");
+    *bytes = part_layout(n_slots, arrival_cap).total;
+    return DBLP_OK;
+}
+
+extern "C" int dblp_aggregate_claim_grouped(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, uint64_t n_slots,
+                                            const uint32_t* arrival, const uint64_t* n_arrived_dev, uint64_t arrival_cap,
+                                            uint32_t round, uint64_t* slot_key, dblp_counters_t* counters, void* ws,
+                                            size_t ws_bytes, void* stream)
+{
+    DBLP_REQUIRE(plan && hdr_ring && arrival && n_arrived_dev && slot_key && counters && ws, DBLP_EINVAL,
+                 "aggregate_claim_grouped: null argument");
+    DBLP_REQUIRE(aligned16(hdr_ring), DBLP_EALIGN, "aggregate_claim_grouped: header ring must be 16-byte aligned");
+    DBLP_REQUIRE((reinterpret_cast<uintptr_t>(ws) & 255u) == 0, DBLP_EALIGN, "aggregate_claim_grouped: workspace must be 256-byte aligned");
+    DBLP_REQUIRE(n_slots < 0xFFFFFFFFull && arrival_cap < (1ull << 32), DBLP_ECAPACITY,
+                 "aggregate_claim_grouped: ring or arrival list too long");
+    if (arrival_cap == 0) return DBLP_OK;
+    const PartLayout l = part_layout(n_slots, arrival_cap);
+    DBLP_REQUIRE(ws_bytes >= l.total, DBLP_ECAPACITY, "aggregate_claim_grouped: workspace of %zu bytes, %zu needed", ws_bytes, l.total);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint8_t* base = static_cast<uint8_t*>(ws);
+    uint2* pairs = reinterpret_cast<uint2*>(base + l.pairs);
+    uint32_t* hist = reinterpret_cast<uint32_t*>(base + l.hist);
+    k_part_count<<<l.n_blocks, kPartThreads, 0, s>>>(arrival, n_arrived_dev, arrival_cap, l.shift, hist);
+    DBLP_LAUNCHED();
+    uint32_t* totals = reinterpret_cast<uint32_t*>(base + l.totals);
+    k_part_offsets<<<kPartBuckets, 1024, 0, s>>>(hist, l.n_blocks, totals);
+    DBLP_LAUNCHED();
+    k_part_scatter<<<l.n_blocks, kPartThreads, 0, s>>>(arrival, n_arrived_dev, arrival_cap, l.shift, hist, totals, pairs);
+    DBLP_LAUNCHED();
+    const unsigned grid = (unsigned)((arrival_cap + kBookThreads * kBookItems - 1) / (kBookThreads * kBookItems));
+    k_book<kBookPairs><<<grid, kBookThreads, 0, s>>>(hdr_ring, n_slots, reinterpret_cast<const uint32_t*>(pairs), n_arrived_dev,
+                                                     arrival_cap, round, reinterpret_cast<unsigned long long*>(slot_key), counters,
+                                                     plan->d_tensor_tab, plan->T, plan->W, plan->C, plan->E, plan->es,
+                                                     plan->hdr_stride, 0, 0);
+    DBLP_LAUNCHED();
+    return DBLP_OK;
+}
 
 extern "C" int dblp_aggregate_claim(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, uint64_t n_slots,
                                     const uint32_t* arrival, const uint64_t* n_arrived_dev, uint64_t arrival_cap,

@@ -122,6 +122,9 @@ struct dblp_plan {
     // dblp_round_reset as one kernel that leaves the claim table in L2 (tables up to a quarter of the L2), instead of
     // three memsets
     uint32_t reset_in_l2;
+    // dblp_round_receive groups the arrivals by slot range before claiming (dblp_aggregate_claim_grouped): chosen when
+    // headers and claim table together exceed the L2
+    uint32_t claim_grouped;
 };
 
 namespace dblp {

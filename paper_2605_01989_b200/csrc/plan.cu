@@ -155,6 +155,7 @@ static int plan_create(const uint64_t* tensor_numel, uint32_t T, int dtype, uint
     DBLP_REQUIRE(e == cudaSuccess, DBLP_ECUDA, "plan: device query failed: %s", cudaGetErrorString(e));
     p->pack_tile_major = p->M * (uint64_t)payload_bytes <= 16ull * (uint64_t)l2_bytes ? 1u : 0u;
     p->reset_in_l2 = p->M * sizeof(uint64_t) <= (uint64_t)l2_bytes / 4 && p->M >= 8 ? 1u : 0u;
+    p->claim_grouped = p->M * (sizeof(dblp_hdr_t) + sizeof(uint64_t)) > (uint64_t)l2_bytes ? 1u : 0u;
     guard.p = nullptr;
     *out = p;
     return DBLP_OK;

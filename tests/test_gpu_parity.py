@@ -142,7 +142,19 @@ def test_sweep_sample_across_every_axis():
         H.full_round_parity(p, flags_list=(dblp.DBLP_MEAN,))
 
 
-def test_stale_duplicate_and_invalid_packets_and_second_attempt():
+def _aggregate(g, rnd, flags, grouped):
+    """dblp_aggregate, or the same with the claims grouped by slot range first."""
+    if not grouped:
+        return g.aggregate(rnd, flags)
+    b = g.buf
+    dblp.dblp_aggregate_claim_grouped(g.plan, b["hdr_ring"], b["n_slots"], b["arrival"], b["n_arrived"], b["arrival_cap"], rnd,
+                                      b["slot_key"], b["counters"], b["ws"])
+    dblp.dblp_aggregate_bitmap(g.plan, b["slot_key"], b["n_arrived"], b["arrival_cap"], b["recv_bitmap"], b["counters"])
+    dblp.dblp_aggregate_reduce(g.plan, b["payload_ring"], b["slot_key"], b["agg"], flags)
+
+
+@pytest.mark.parametrize("grouped", [False, True], ids=["claims in arrival order", "claims grouped by slot range"])
+def test_stale_duplicate_and_invalid_packets_and_second_attempt(grouped):
     w = work(RAGGED, "f32", 1408, 4, wl.LossSpec("iid", 0.3), 21)
     rnd = w.round
     grads = wl.make_grads(w, H.DEV)
@@ -190,7 +202,7 @@ def test_stale_duplicate_and_invalid_packets_and_second_attempt():
     rng.shuffle(mixed)
     g.buf["arrival"][:len(mixed)].copy_(torch.from_numpy(mixed.view(np.int32)))
     g.buf["n_arrived"].fill_(len(mixed))
-    g.aggregate(rnd)
+    _aggregate(g, rnd, dblp.DBLP_SUM, grouped)
     st = op.book(o_hdr2, mixed, len(mixed), rnd, op.new_state())
     c = st["counters"].as_dict()
     assert c["n_stale"] > 50 and c["n_dup"] > 50 and c["n_invalid"] > 100
@@ -202,13 +214,45 @@ def test_stale_duplicate_and_invalid_packets_and_second_attempt():
     o_del1, _ = op.loss_mask(om, w.seed, rnd, attempt=1)
     o_arr1, o_n1 = op.arrival(o_del1, w.seed, rnd, attempt=1)
     H.assert_bits_equal(H.u32(g.buf["arrival"])[:o_n1], o_arr1[:o_n1], "arrival list, attempt 1")
-    g.aggregate(rnd, dblp.DBLP_MEAN)
+    _aggregate(g, rnd, dblp.DBLP_MEAN, grouped)
     st = op.book(o_hdr2, o_arr1, o_n1, rnd, st)
     H.compare_state(g, st, op)
     H.assert_bits_equal(g.buf["agg"].cpu().numpy(), op.reduce(o_pay2, st, mean=True), "aggregate after attempt 1")
     assert st["counters"].as_dict()["n_dup"] > c["n_dup"]
     H.compare_bound(g, op, st["bitmap"], 100000)
     g.close()
+
+
+@pytest.mark.parametrize("C", [1, 63, 64, 65, 4097, 70001])
+def test_grouped_claims_leave_the_same_table_as_plain_claims(C):
+    """Ring sizes around the limits of the grouping (fewer slots than ranges, one more than a power of two times the
+    range count), with repeats and out-of-ring entries in the arrival list: claim table, bitmap and counters must be
+    identical, byte for byte, to those of dblp_aggregate_claim."""
+    w = work([C * 4], "f32", 16, 3, wl.LossSpec("iid", 0.2), 5 + C)
+    grads = wl.make_grads(w, H.DEV)
+    a, b = H.GpuRound(w, arrival_cap=2 * 3 * C + 8), H.GpuRound(w, arrival_cap=2 * 3 * C + 8)
+    gm, _ = H.models_for(w, a.plan.C)
+    M = a.plan.M
+    rng = np.random.default_rng(C)
+    for attempt in range(2):                             # the second call continues the arrival numbers of the first
+        for g in (a, b):
+            g.packetize(grads, w.round)
+            g.apply_loss(gm, w.seed, w.round, attempt)
+        n = a.n_arrived()
+        extra = np.concatenate([rng.integers(0, M, n // 3 + 1), [M, M + 7, 0xFFFFFFFF]]).astype(np.uint32)
+        mixed = np.concatenate([H.u32(a.buf["arrival"])[:n], extra])
+        rng.shuffle(mixed)
+        for g in (a, b):
+            g.buf["arrival"][:len(mixed)].copy_(torch.from_numpy(mixed.view(np.int32)))
+            g.buf["n_arrived"].fill_(len(mixed))
+        _aggregate(a, w.round, dblp.DBLP_SUM, False)
+        _aggregate(b, w.round, dblp.DBLP_SUM, True)
+        torch.cuda.synchronize()
+        for name in ("slot_key", "recv_bitmap", "counters", "agg"):
+            assert torch.equal(a.buf[name].view(torch.uint8), b.buf[name].view(torch.uint8)), (name, attempt)
+        assert dblp.counters_dict(b.buf["counters"])["n_invalid"] == 3 * (attempt + 1)
+    a.close()
+    b.close()
 
 
 def test_physically_permuted_ring():
