@@ -233,16 +233,28 @@ __global__ void __launch_bounds__(kPartThreads)
 k_part_count(const uint32_t* __restrict__ arrival, const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap,
              uint32_t shift, uint32_t* __restrict__ block_hist)
 {
-    __shared__ uint32_t s_hist[kPartBuckets];
-    if (threadIdx.x < kPartBuckets) s_hist[threadIdx.x] = 0;
+    constexpr int kWarps = kPartThreads / 32;
+    __shared__ uint32_t s_hist[kWarps][kPartBuckets];               // one histogram per warp: fewer colliding atomics
+    for (uint32_t k = threadIdx.x; k < kWarps * kPartBuckets; k += kPartThreads) (&s_hist[0][0])[k] = 0;
     __syncthreads();
     const uint64_t n = min(*n_arrived_dev, arrival_cap), base = (uint64_t)blockIdx.x * kPartChunk;
-    for (uint32_t k = threadIdx.x; k < kPartChunk; k += kPartThreads) {
-        const uint64_t a = base + k;
-        if (a < n) atomicAdd(&s_hist[part_bucket(__ldg(&arrival[a]), shift)], 1u);
+    uint32_t* mine = s_hist[threadIdx.x >> 5];
+    constexpr int kPer = kPartChunk / kPartThreads;
+    uint32_t slot[kPer];
+#pragma unroll
+    for (int k = 0; k < kPer; ++k) {                                // all loads first, so that they are in flight together
+        const uint64_t a = base + threadIdx.x + (uint64_t)k * kPartThreads;
+        slot[k] = a < n ? __ldg(&arrival[a]) : 0u;
     }
+#pragma unroll
+    for (int k = 0; k < kPer; ++k)
+        if (base + threadIdx.x + (uint64_t)k * kPartThreads < n) atomicAdd(&mine[part_bucket(slot[k], shift)], 1u);
     __syncthreads();
-    if (threadIdx.x < kPartBuckets) block_hist[(uint64_t)threadIdx.x * gridDim.x + blockIdx.x] = s_hist[threadIdx.x];   // [range][block]
+    if (threadIdx.x < kPartBuckets) {
+        uint32_t t = 0;
+        for (int w = 0; w < kWarps; ++w) t += s_hist[w][threadIdx.x];
+        block_hist[(uint64_t)threadIdx.x * gridDim.x + blockIdx.x] = t;   // [range][block]
+    }
 }
 
 // One block per range: the range's per-block counts (a contiguous row of the table) become exclusive prefix sums, and
@@ -273,26 +285,54 @@ k_part_offsets(uint32_t* __restrict__ block_hist, uint32_t n_blocks, uint32_t* _
     if (threadIdx.x == 1023) range_total[blockIdx.x] = s_scan[1023];
 }
 
+// The block first sorts its kPartChunk entries by range in shared memory (a local counting sort), then copies each
+// range's run to its place in the pair list, so that the global stores are runs of consecutive pairs instead of single
+// 8-byte stores all over the list.
 __global__ void __launch_bounds__(kPartThreads)
 k_part_scatter(const uint32_t* __restrict__ arrival, const uint64_t* __restrict__ n_arrived_dev, uint64_t arrival_cap,
                uint32_t shift, const uint32_t* __restrict__ block_off, const uint32_t* __restrict__ range_total,
                uint2* __restrict__ pairs)
 {
-    __shared__ uint32_t s_cursor[kPartBuckets];
+    constexpr int kPer = kPartChunk / kPartThreads;
+    __shared__ uint2 s_pairs[kPartChunk];
+    __shared__ uint32_t s_count[kPartBuckets], s_start[kPartBuckets], s_global[kPartBuckets];
     if (threadIdx.x < kPartBuckets) {
         uint32_t first = 0;                                          // where this thread's range starts in the pair list
-        for (uint32_t b = 0; b < threadIdx.x; ++b) first += __ldg(&range_total[b]);
-        s_cursor[threadIdx.x] = first + block_off[(uint64_t)threadIdx.x * gridDim.x + blockIdx.x];
+        for (uint32_t r = 0; r < threadIdx.x; ++r) first += __ldg(&range_total[r]);
+        s_global[threadIdx.x] = first + block_off[(uint64_t)threadIdx.x * gridDim.x + blockIdx.x];
+        s_count[threadIdx.x] = 0;
     }
     __syncthreads();
     const uint64_t n = min(*n_arrived_dev, arrival_cap), base = (uint64_t)blockIdx.x * kPartChunk;
-    for (uint32_t k = threadIdx.x; k < kPartChunk; k += kPartThreads) {
-        const uint64_t a = base + k;
-        if (a < n) {
-            const uint32_t slot = __ldg(&arrival[a]);
-            const uint32_t at = atomicAdd(&s_cursor[part_bucket(slot, shift)], 1u);
-            pairs[at] = make_uint2(slot, (uint32_t)a);
-        }
+    uint32_t slot[kPer], rank[kPer];
+#pragma unroll
+    for (int k = 0; k < kPer; ++k) {                                // all loads first, so that they are in flight together
+        const uint64_t a = base + threadIdx.x + (uint64_t)k * kPartThreads;
+        slot[k] = a < n ? __ldg(&arrival[a]) : 0u;
+    }
+#pragma unroll
+    for (int k = 0; k < kPer; ++k) {
+        const uint64_t a = base + threadIdx.x + (uint64_t)k * kPartThreads;
+        rank[k] = a < n ? atomicAdd(&s_count[part_bucket(slot[k], shift)], 1u) : kEmpty32;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t run = 0;
+        for (int r = 0; r < kPartBuckets; ++r) { s_start[r] = run; run += s_count[r]; }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < kPer; ++k)
+        if (rank[k] != kEmpty32)
+            s_pairs[s_start[part_bucket(slot[k], shift)] + rank[k]] =
+                make_uint2(slot[k], (uint32_t)(base + threadIdx.x + (uint64_t)k * kPartThreads));
+    __syncthreads();
+    const uint64_t left = n > base ? n - base : 0;
+    const uint32_t have = left < (uint64_t)kPartChunk ? (uint32_t)left : (uint32_t)kPartChunk;
+    for (uint32_t i = threadIdx.x; i < have; i += kPartThreads) {
+        const uint2 pr = s_pairs[i];
+        const uint32_t r = part_bucket(pr.x, shift);
+        pairs[s_global[r] + (i - s_start[r])] = pr;
     }
 }
 
