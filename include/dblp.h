@@ -229,9 +229,12 @@ int dblp_aggregate_claim(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, ui
  * slot range (a counting sort in three small passes into (position, slot) pairs in ws), then the claims are made range
  * by range, so that the headers and cells they touch stay in L2 instead of costing two random DRAM sectors per packet;
  * a packet's arrival number travels with it, so "first arrival wins" is unchanged.  On 12 M packets the claim stage
- * drops from 0.54 to 0.25 ms; below a few million packets dblp_aggregate_claim is the faster one (dblp_round_receive
- * chooses by the plan's size).  ws: dblp_claim_workspace_bytes(n_slots, arrival_cap) bytes, 256-byte aligned, contents
- * need not be preserved. */
+ * drops from 0.53 to 0.29 ms; below about 3 M packets the plain order is the faster one.
+ * dblp_aggregate_claim chooses by itself: a plan whose headers and claim table exceed the L2 owns a scratch of
+ * dblp_claim_workspace_bytes(M, M) bytes (allocated in dblp_plan_create, 8 bytes per packet) and groups every call
+ * with n_slots <= M and arrival_cap <= M; such a plan serves one claim at a time.  This entry point is for callers who
+ * want the grouping elsewhere or with a scratch of their own.  ws: dblp_claim_workspace_bytes(n_slots, arrival_cap)
+ * bytes, 256-byte aligned, contents need not be preserved. */
 int dblp_claim_workspace_bytes(const dblp_plan_t* plan, uint64_t n_slots, uint64_t arrival_cap, size_t* bytes);
 int dblp_aggregate_claim_grouped(const dblp_plan_t* plan, const dblp_hdr_t* hdr_ring, uint64_t n_slots,
                                  const uint32_t* arrival, const uint64_t* n_arrived_dev, uint64_t arrival_cap,
@@ -332,8 +335,7 @@ typedef struct {
     uint32_t* missing_cnt;     /* W * B */
     uint8_t* ok;               /* W * B */
     uint32_t* all_ok;          /* 1 */
-    void* ws;                  /* dblp_workspace_bytes; max with dblp_claim_workspace_bytes(M, M) to let large rounds group
-                                  their claims, and with dblp_stop_workspace_bytes(M) for dblp_round_until_stop */
+    void* ws;                  /* dblp_workspace_bytes (max with dblp_stop_workspace_bytes(M) for dblp_round_until_stop) */
     size_t ws_bytes;
     uint32_t* sent_bits;       /* W * row_words; used by dblp_round_until_stop only */
 } dblp_device_buffers_t;
@@ -358,8 +360,7 @@ typedef struct {
  * every worker, then the mean; Algorithm 2 inside; Section III-B for the tolerance test):
  *   dblp_round_send     round_reset and apply_loss (attempt 0) on the plan's side stream beside dblp_packetize on the
  *                       caller's stream; returns with the caller's stream waiting for both.
- *   dblp_round_receive  dblp_aggregate_claim (dblp_aggregate_claim_grouped for rounds of several million packets, when
- *                       dev->ws is large enough for it), then dblp_aggregate_bitmap + dblp_check_bound (one tolerance for all) on
+ *   dblp_round_receive  dblp_aggregate_claim, then dblp_aggregate_bitmap + dblp_check_bound (one tolerance for all) on
  *                       the side stream beside dblp_aggregate_reduce; the caller's stream waits for both at the end.
  * grads: HOST array of W device pointers as for dblp_packetize.  flags: DBLP_SUM or DBLP_MEAN.  Packets occupy ring slots
  * 0 .. M-1.  Nothing is allocated and the host is not blocked.  The side stream and its events belong to the plan, so a

@@ -1265,6 +1265,10 @@ extern "C" int dblp_aggregate_claim(const dblp_plan_t* plan, const dblp_hdr_t* h
                                     const uint32_t* arrival, const uint64_t* n_arrived_dev, uint64_t arrival_cap,
                                     uint32_t round, uint64_t* slot_key, dblp_counters_t* counters, void* stream)
 {
+    // rounds whose headers and claim table exceed L2: grouped by slot range first, in the plan's own scratch
+    if (plan && plan->claim_grouped && plan->d_claim_ws && n_slots <= plan->M && arrival_cap <= plan->M)
+        return dblp_aggregate_claim_grouped(plan, hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, slot_key,
+                                            counters, plan->d_claim_ws, plan->claim_ws_bytes, stream);
     return claim_arrivals(plan, hdr_ring, n_slots, arrival, n_arrived_dev, arrival_cap, round, slot_key, counters, 0, 0,
                           static_cast<cudaStream_t>(stream));
 }

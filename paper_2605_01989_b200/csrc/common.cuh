@@ -125,6 +125,8 @@ struct dblp_plan {
     // dblp_round_receive groups the arrivals by slot range before claiming (dblp_aggregate_claim_grouped): chosen when
     // headers and claim table together exceed the L2
     uint32_t claim_grouped;
+    void* d_claim_ws;       // scratch of the grouped claims (dblp_claim_workspace_bytes(M, M) bytes); null unless claim_grouped
+    size_t claim_ws_bytes;
 };
 
 namespace dblp {

@@ -30,6 +30,7 @@ static void free_tables(dblp_plan* p)
     cudaFree(p->d_bucket_bounds);
     cudaFree(p->d_bound_ppm);
     cudaFree(p->d_ticket);
+    cudaFree(p->d_claim_ws);
     if (p->side) cudaStreamDestroy(p->side);
     if (p->copy) cudaStreamDestroy(p->copy);
     if (p->back) cudaStreamDestroy(p->back);
@@ -91,6 +92,7 @@ static int plan_create(const uint64_t* tensor_numel, uint32_t T, int dtype, uint
     p->hdr_stride = 32; p->pay_stride = payload_bytes; p->pay_off = 0;
     p->d_tensor_tab = nullptr; p->d_base = nullptr; p->d_chunk_desc = nullptr;
     p->d_chunk_tensor = p->d_bucket_bounds = p->d_bound_ppm = p->d_ticket = nullptr;
+    p->d_claim_ws = nullptr; p->claim_ws_bytes = 0;
     p->side = p->copy = p->back = nullptr;
     p->ev_fork = p->ev_join = p->ev_claimed = p->ev_done = p->ev_copy[0] = p->ev_copy[1] = nullptr;
     p->ev_part[0] = p->ev_part[1] = p->ev_back = nullptr;
@@ -156,6 +158,13 @@ static int plan_create(const uint64_t* tensor_numel, uint32_t T, int dtype, uint
     p->pack_tile_major = p->M * (uint64_t)payload_bytes <= 16ull * (uint64_t)l2_bytes ? 1u : 0u;
     p->reset_in_l2 = p->M * sizeof(uint64_t) <= (uint64_t)l2_bytes / 4 && p->M >= 8 ? 1u : 0u;
     p->claim_grouped = p->M * (sizeof(dblp_hdr_t) + sizeof(uint64_t)) > (uint64_t)l2_bytes ? 1u : 0u;
+    if (p->claim_grouped) {                                         // 8 bytes per packet, e.g. 97 MB for 12 M packets
+        const int rcw = dblp_claim_workspace_bytes(p, p->M, p->M, &p->claim_ws_bytes);
+        if (rcw != DBLP_OK) return rcw;
+        e = cudaMalloc(&p->d_claim_ws, p->claim_ws_bytes);
+        DBLP_REQUIRE(e == cudaSuccess, DBLP_ECUDA, "plan: scratch of the grouped claims (%zu bytes): %s", p->claim_ws_bytes,
+                     cudaGetErrorString(e));
+    }
     guard.p = nullptr;
     *out = p;
     return DBLP_OK;

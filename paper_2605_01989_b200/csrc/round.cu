@@ -76,14 +76,8 @@ extern "C" int dblp_round_receive(const dblp_plan_t* plan, uint32_t round, uint3
     DBLP_TRY(check_buffers(dev, "round_receive"));
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     DBLP_TRY(mark(marks ? marks->receive_begin : nullptr, s));
-    size_t grouped_ws = 0;
-    if (plan->claim_grouped) DBLP_TRY(dblp_claim_workspace_bytes(plan, plan->M, plan->M, &grouped_ws));
-    if (plan->claim_grouped && dev->ws_bytes >= grouped_ws)         // the loss process is done with the workspace by now
-        DBLP_TRY(dblp_aggregate_claim_grouped(plan, dev->hdr_ring, plan->M, dev->arrival, dev->n_arrived, plan->M, round,
-                                              dev->slot_key, dev->counters, dev->ws, dev->ws_bytes, s));
-    else
-        DBLP_TRY(dblp_aggregate_claim(plan, dev->hdr_ring, plan->M, dev->arrival, dev->n_arrived, plan->M, round,
-                                      dev->slot_key, dev->counters, s));
+    DBLP_TRY(dblp_aggregate_claim(plan, dev->hdr_ring, plan->M, dev->arrival, dev->n_arrived, plan->M, round, dev->slot_key,
+                                  dev->counters, s));
     DBLP_TRY(mark(marks ? marks->claim_end : nullptr, s));
     DBLP_CUDA(cudaEventRecord(plan->ev_claimed, s));
     DBLP_CUDA(cudaStreamWaitEvent(plan->side, plan->ev_claimed, 0));
