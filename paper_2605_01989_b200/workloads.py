@@ -131,8 +131,8 @@ class Workload:
         return self.W * self.C
 
     def device_bytes(self) -> int:
-        """Gradients + payload ring + fp32 aggregate + per-packet metadata."""
-        return self.W * self.N * self.elem_size + self.M * self.payload_bytes + self.N * 4 + self.M * (32 + 4 + 8)
+        """Gradients + payload ring + fp32 aggregate + per-packet metadata and scratch."""
+        return self.W * self.N * self.elem_size + self.M * self.payload_bytes + self.N * 4 + self.M * (32 + 4 + 8 + 8 + 8)
 
 
 def config(i: int) -> Workload:
